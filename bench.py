@@ -1,0 +1,379 @@
+"""Benchmark of the append-prefill hot path of one sparse layer: indexer -> top-k -> page demand -> sparse attention.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic session (the exact pass; the predicted pass that feeds the
+miss set is prepared once, untimed).  Metric: new tokens/s per sparse layer.  Prints ONE JSON line (rank 0).
+With N > 1 (torchrun) every rank runs its own session (independent problems, no data-path collective): weak scaling.
+--impl reference times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "append_prefill_new_tokens_per_sec_per_sparse_layer"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def workload_numbers(shp):
+    """Algorithmic work of one step (exact pass), per the definitions in the design doc."""
+    L, M, S = shp.L, shp.M, shp.S
+    pairs = M * L + M * (M + 1) // 2
+    sel = sum(min(shp.k, L + t + 1) for t in range(M))
+    esz = 2 if shp.idx_dtype == "bf16" else 1
+    row_bytes = shp.d_qk * 2 if shp.attn == "latent" else (shp.d_qk + shp.d_v) * 2 * shp.n_kv_heads
+    return {
+        "pairs": pairs,
+        "indexer_flops": 2.0 * shp.H_I * shp.D_I * pairs,
+        "indexer_bytes": esz * (M * shp.H_I * shp.D_I + S * shp.D_I) + 4 * M * shp.H_I + 4.0 * pairs,
+        "topk_bytes": 4.0 * pairs + 4.0 * M * shp.k,
+        "page_demand_bytes": 4.0 * M * shp.k,
+        "attn_flops": 2.0 * shp.H_q * (shp.d_qk + shp.d_v) * sel,
+        "attn_bytes": float(row_bytes) * sel + 2.0 * M * shp.H_q * (shp.d_qk + shp.d_v),
+        "selected_rows": sel,
+    }
+
+
+def run_reference(args, shp, sess):
+    """The CPU oracle, as it stands, on a bounded sample of query rows of the same workload."""
+    from oracle import janus_oracle as O
+    from paper_2609_36938_b200 import workloads as W
+
+    n_rows = args.ref_rows
+    rows = W.sample_rows(shp.M, n_rows)
+
+    def step():
+        sc = O.indexer_scores(sess["q_idx"], sess["k_idx"], sess["w"], dtype=shp.idx_dtype, q_scale=sess["q_scale"], k_scale=sess["k_scale"],
+                              recency=sess["recency"], q_pos0=shp.L, causal=True, rows=rows)
+        idx = O.topk(sc, shp.k, q_pos0=shp.L, causal=True, rows=rows)
+        O.page_demand(idx, shp.L, shp.page_size, sess["page_table"])
+        O.sparse_attention(sess["Q"], sess["k_pool"], sess["v_pool"], sess["page_table"], idx, page_size=shp.page_size,
+                           softmax_scale=shp.softmax_scale, d_qk=shp.d_qk, d_v=shp.d_v, rows=rows)
+
+    for _ in range(args.warmup_ref):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps_ref):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps_ref
+    cores = len(os.sched_getaffinity(0))
+    value = len(rows) / dt
+    return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(rows)} of {shp.M} query rows (first, last, evenly spread), all {shp.S} keys, k={shp.k}; "
+                      f"rows are independent, rows/s reported as tokens/s", "ms_per_step": dt * 1e3}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, help="benchmark configuration 1..5 (4 = first session of the ragged batch)")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--L", type=int, default=None)
+    ap.add_argument("--M", type=int, default=None)
+    ap.add_argument("--ref-rows", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    args.steps_ref = max(1, min(args.steps, 3))
+    args.warmup_ref = 1 if args.warmup > 0 else 0
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2609_36938_b200 import workloads as W
+
+    if args.workload == 4:
+        shp = W.batch_shapes(args.seed)[0]
+    else:
+        shp = W.config_shape(args.workload, L=args.L, M=args.M)
+    workload_name = (f"config {args.workload}: L={shp.L} M={shp.M} k={shp.k}, indexer {shp.H_I}x{shp.D_I} {shp.idx_dtype}, "
+                     f"{shp.attn} attention {shp.H_q} heads {shp.d_qk}/{shp.d_v} bf16, page {shp.page_size}, {shp.table} page table")
+    config = {"workload": workload_name, "sessions_per_gpu": 1, "cache": "inputs larger than L2 (scores, Q and gathered KV are GBs per step)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        sess = W.make_session(shp, args.seed)
+        cb = run_reference(args, shp, sess)
+        line = {"metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps_ref, "warmup": args.warmup_ref,
+                "ms_per_step": cb["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": config, "impl": "reference",
+                "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_36938_b200 import binding as B, build as _build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    B.load()
+
+    sess = W.make_session(shp, args.seed + rank)
+    kind = shp.idx_dtype
+    host = {
+        "q_idx": (sess["q_idx"], kind), "k_idx": (sess["k_idx"], kind), "w": (sess["w"], "f32"), "q_scale": (sess["q_scale"], "f32"),
+        "k_scale": (sess["k_scale"], "f32"), "row_bias": (sess["row_bias"], "f32"), "col_bias": (sess["col_bias"], "f32"),
+        "page_table": (sess["page_table"], "i32"), "Q": (sess["Q"], "bf16"), "k_pool": (sess["k_pool"], "bf16"),
+    }
+    if sess["v_pool"] is not sess["k_pool"]:
+        host["v_pool"] = (sess["v_pool"], "bf16")
+    pinned = {}
+    for name, (arr, kd) in host.items():
+        if arr is None:
+            pinned[name] = None
+            continue
+        t = B.to_device(arr, kd, device="cpu")
+        pinned[name] = t.pin_memory()
+    h2d_bytes = sum(t.numel() * t.element_size() for t in pinned.values() if t is not None)
+
+    def upload():
+        d = {n: (None if t is None else t.to("cuda", non_blocking=True)) for n, t in pinned.items()}
+        if "v_pool" not in d:
+            d["v_pool"] = d["k_pool"]
+        return d
+
+    d = upload()
+    n_phys = sess["n_phys_pages"]
+    ld = (shp.S + 31) // 32 * 32
+    scores = torch.empty((shp.M, ld), dtype=torch.float32, device="cuda")
+    out_buf = torch.empty((shp.M, shp.H_q, shp.d_v), dtype=torch.bfloat16, device="cuda")
+
+    # predicted pass (Eq. 2): same indexer on the lookahead queries over the history keys only; prepared once
+    pred_bitmap = None
+    if "q_pred" in sess:
+        qp = B.to_device(sess["q_pred"], kind)
+        psc = B.janus_indexer_scores(qp, d["k_idx"][:shp.L], d["w"], q_scale=d["q_scale"],
+                                     k_scale=None if d["k_scale"] is None else d["k_scale"][:shp.L], q_pos0=shp.L, causal=False)
+        pidx, _, _ = B.janus_topk(psc, shp.L, shp.k, q_pos0=shp.L, causal=False, want_count=False, want_kth=False)
+        pred_bitmap = B.janus_page_demand(pidx, demand_limit=shp.L, page_size=shp.page_size, page_table=d["page_table"],
+                                          n_phys_pages=n_phys, want_miss=False)["bitmap"]
+        del psc, pidx, qp
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    stream = torch.cuda.current_stream()
+
+    def step(d, marks=None):
+        if marks is not None:
+            marks[0].record(stream)
+        sc = B.janus_indexer_scores(d["q_idx"], d["k_idx"], d["w"], q_scale=d["q_scale"], k_scale=d["k_scale"], row_bias=d["row_bias"],
+                                    col_bias=d["col_bias"], q_pos0=shp.L, causal=True, scores=scores)
+        if marks is not None:
+            marks[1].record(stream)
+        idx, _, _ = B.janus_topk(sc, shp.S, shp.k, q_pos0=shp.L, causal=True, want_count=False, want_kth=False)
+        if marks is not None:
+            marks[2].record(stream)
+        pd = B.janus_page_demand(idx, demand_limit=shp.L, page_size=shp.page_size, page_table=d["page_table"], n_phys_pages=n_phys,
+                                 predicted_bitmap=pred_bitmap)
+        if marks is not None:
+            marks[3].record(stream)
+        out, _ = B.janus_sparse_attn_prefill(d["Q"], d["k_pool"], d["v_pool"], idx, page_table=d["page_table"], page_size=shp.page_size,
+                                             softmax_scale=shp.softmax_scale, d_v=shp.d_v, want_lse=False, out=out_buf)
+        if marks is not None:
+            marks[4].record(stream)
+        return idx, pd, out
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(d)
+    B.check_dev_status()
+
+    # ---- timed region: device-resident inputs
+    marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_start, t_end = ev(), ev()
+    t_start.record(stream)
+    for i in range(args.steps):
+        idx, pd, out = step(d, marks[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    B.check_dev_status()
+    elapsed_ms = t_start.elapsed_time(t_end)
+    per_call = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])   # [steps, 4] ms
+    if world > 1:
+        tt = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * shp.M / (ms_per_step * 1e-3)
+
+    # ---- end to end: every step uploads all inputs from pinned host memory and reads the results back
+    e2e = None
+    if not args.no_e2e:
+        host_out = torch.empty(out_buf.shape, dtype=out_buf.dtype).pin_memory()
+        host_idx = torch.empty((shp.M, shp.k), dtype=torch.int32).pin_memory()
+        host_pages = torch.empty((n_phys,), dtype=torch.int32).pin_memory()
+        host_counts = torch.empty((4,), dtype=torch.int32).pin_memory()
+        d2h_bytes = sum(t.numel() * t.element_size() for t in (host_out, host_idx, host_pages, host_counts))
+
+        def e2e_step():
+            dd = upload()
+            idx, pd, out = step(dd)
+            host_out.copy_(out, non_blocking=True)
+            host_idx.copy_(idx, non_blocking=True)
+            host_pages.copy_(pd["pages"][:n_phys], non_blocking=True)
+            host_counts.copy_(pd["counts"], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        n_e2e = max(2, min(args.steps, 5))
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        if world > 1:
+            tt = torch.tensor([e2e_ms], device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        e2e = {"value": world * shp.M / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
+               "ms_per_step": e2e_ms, "inputs": "all operands (queries, keys, weights, Q, KV pool, page table) uploaded every step"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    wn = workload_numbers(shp)
+    mean_ms = per_call.mean(axis=0)
+    names = ["indexer_scores", "topk", "page_demand", "sparse_attn_prefill"]
+    fp8 = shp.idx_dtype == "fp8"
+    tensor_peak_idx = peaks["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)
+    kernels = {
+        "indexer_scores": {"ms": mean_ms[0], "tflops": wn["indexer_flops"] / (mean_ms[0] * 1e-3) / 1e12,
+                           "frac_tensor_peak": wn["indexer_flops"] / (mean_ms[0] * 1e-3) / 1e12 / tensor_peak_idx},
+        "topk": {"ms": mean_ms[1], "gbs": wn["topk_bytes"] / (mean_ms[1] * 1e-3) / 1e9,
+                 "frac_hbm_peak": wn["topk_bytes"] / (mean_ms[1] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "page_demand": {"ms": mean_ms[2], "gbs": wn["page_demand_bytes"] / (mean_ms[2] * 1e-3) / 1e9},
+        "sparse_attn_prefill": {"ms": mean_ms[3], "tflops": wn["attn_flops"] / (mean_ms[3] * 1e-3) / 1e12,
+                                "logical_gbs": wn["attn_bytes"] / (mean_ms[3] * 1e-3) / 1e9,
+                                "frac_hbm_peak": wn["attn_bytes"] / (mean_ms[3] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "frac_tensor_peak": wn["attn_flops"] / (mean_ms[3] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
+    }
+    dom = int(np.argmax(mean_ms))
+    if names[dom] == "indexer_scores":
+        roofline = {"kernel": "indexer_tc_kernel", "bound": "tensor", "achieved": kernels["indexer_scores"]["tflops"], "peak": tensor_peak_idx,
+                    "unit": "TFLOP/s", "frac": kernels["indexer_scores"]["frac_tensor_peak"], "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 sustained" + (" x2 (nominal fp8:bf16 ratio)" if fp8 else "")}
+    elif names[dom] == "sparse_attn_prefill":
+        roofline = {"kernel": "sparse_attn", "bound": "tensor", "achieved": kernels["sparse_attn_prefill"]["tflops"],
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": kernels["sparse_attn_prefill"]["frac_tensor_peak"],
+                    "traffic": None, "peak_source": f"{peaks['source']} bf16 sustained"}
+    else:
+        key = names[dom]
+        roofline = {"kernel": key, "bound": "hbm", "achieved": kernels[key]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": kernels[key]["gbs"] / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth"}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        cb = run_reference(args, shp, sess)
+        cpu_baseline = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    counts = pd["counts"].cpu().numpy()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3+bf16" if fp8 else "bf16", "data": "synthetic",
+        "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "kernels": {k: {kk: (round(float(vv), 4)) for kk, vv in v.items()} for k, v in kernels.items()},
+        "page_demand": {"n_pages": int(counts[0]), "n_runs": int(counts[1]), "n_miss": int(counts[2]), "n_miss_runs": int(counts[3])},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,171 @@
+/*
+ * janus.h - C boundary of the B200 append-prefill library for top-k sparse-attention layers.
+ *
+ * One sparse layer of an append prefill runs, for the M newly appended tokens of a session with L cached
+ * history tokens (S = L + M keys; the paper's P and L, Table 1):
+ *
+ *     janus_indexer_scores -> janus_topk -> janus_page_demand -> janus_sparse_attn_prefill
+ *
+ * Conventions (all entry points)
+ *   - plain C ABI, no exceptions; every function returns an int status (JANUS_OK or JANUS_ERR_*).
+ *   - every data pointer is a DEVICE pointer owned by the caller, unless a comment says "host".
+ *     The library never allocates or frees device memory; scratch, where a call needs it, is the
+ *     caller's `ws` buffer of at least janus_<fn>_workspace_size(...) bytes (may be NULL when 0).
+ *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - host-detectable problems (NULL pointer, bad size, misalignment, unsupported shape) return an
+ *     error code and launch nothing.
+ *   - conditions only visible on the device (index out of range, output capacity exceeded, a bounded
+ *     wait that gave up) are written to *dev_status (first error wins; 0 = none) and the offending
+ *     element is skipped; nothing traps.  dev_status may be NULL.  The caller zeroes it.
+ *   - positions, token indices and page ids are 0-based.  Padding in index arrays is -1.
+ */
+#ifndef JANUS_H_
+#define JANUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host return codes */
+#define JANUS_OK 0
+#define JANUS_ERR_INVALID_ARG 1         /* NULL/negative/misaligned argument                      */
+#define JANUS_ERR_UNSUPPORTED 2         /* shape or dtype combination has no kernel               */
+#define JANUS_ERR_WORKSPACE_TOO_SMALL 3
+#define JANUS_ERR_CUDA 4                /* a CUDA call failed; see janus_last_cuda_error()        */
+
+/* values written to *dev_status by kernels */
+#define JANUS_DEV_OK 0
+#define JANUS_DEV_INDEX_OUT_OF_RANGE 101   /* a token index or page id outside its table (skipped)   */
+#define JANUS_DEV_CAPACITY_EXCEEDED 102    /* more pages/runs than `capacity`; counts are still true */
+#define JANUS_DEV_WAIT_TIMEOUT 103         /* a bounded in-kernel wait gave up; output is incomplete */
+
+/* dtype of the indexer operands */
+#define JANUS_DTYPE_BF16 0
+#define JANUS_DTYPE_FP8_E4M3 1
+
+/* Library version (major*10000 + minor*100 + patch). */
+int janus_version(void);
+
+/* cudaError_t of the most recent failed CUDA call made by this library on the calling thread (0 if none). */
+int janus_last_cuda_error(void);
+
+/*
+ * Indexer scores - the scoring half of Eq. 1 (Sec. 2.2): relevance of every visible token for each new token.
+ * The paper leaves the scoring function to the model reports; this library computes, in fp32 accumulation,
+ *
+ *     scores[t, s] = sum_{h < H_I} w[t, h] * max(0, < q_idx[t, h, :], k_idx[s, :] >)  (+ row_bias[t] * col_bias[s])
+ *
+ * for s <= q_pos0 + t when `causal` (the token itself included), for every s < n_keys otherwise; masked entries
+ * are written as -inf.  One indexer key per token is shared by all indexer heads.
+ *
+ *   q_idx        [M, H_I, D_I]   bf16 or E4M3 bytes; token stride q_stride_tok elements (>= H_I*D_I), heads contiguous
+ *   k_idx        [n_keys, D_I]   same dtype; token stride k_stride_tok elements
+ *   w            [M, H_I]        fp32, any sign
+ *   q_scale      FP8 only: per-head scales [H_I] (q_scale_stride_tok = 0) or per (token, head) [M, H_I]
+ *                (q_scale_stride_tok = H_I); every scale > 0.  NULL for bf16.  True query = e4m3 * q_scale.
+ *   k_scale      FP8 only: per-key scales [n_keys], every scale > 0.  NULL for bf16.
+ *   row_bias, col_bias  optional rank-1 additive term, both NULL or both given ([M] and [n_keys] fp32).
+ *   q_pos0       position of new token 0 among the keys (= L for an append prefill over history + new tokens)
+ *   scores       [M, scores_ld] fp32 out, scores_ld >= n_keys and a multiple of 4; columns >= n_keys untouched
+ *
+ * D_I must be a multiple of 16.  Pointers must be 16-byte aligned; strides multiples of 16 bytes.
+ * The tensor-core kernel serves H_I in {4, 8, 16, 32, 64} with D_I in {64, 128} and dense q_idx
+ * (q_stride_tok == H_I*D_I); other shapes run a slower general kernel.
+ */
+size_t janus_indexer_scores_workspace_size(int M, int H_I, int D_I, int64_t n_keys, int dtype);
+int janus_indexer_scores(const void* q_idx, int64_t q_stride_tok,
+                         const void* k_idx, int64_t k_stride_tok,
+                         const float* w,
+                         const float* q_scale, int64_t q_scale_stride_tok,
+                         const float* k_scale,
+                         const float* row_bias, const float* col_bias,
+                         int M, int H_I, int D_I, int64_t n_keys,
+                         int64_t q_pos0, int causal, int dtype,
+                         float* scores, int64_t scores_ld,
+                         void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Per-row top-k - the selection half of Eq. 1 (Sec. 2.2): for each new token, the indices of its
+ * min(k, prefix) highest-scoring visible keys, prefix = min(n_keys, q_pos0 + t + 1) when causal, else n_keys.
+ * Only scores[t, 0:prefix] is read.  Ties at the threshold are broken arbitrarily; output order is
+ * unspecified; unused slots are -1.  NaN scores are not supported.
+ *
+ *   scores  [M, scores_ld] fp32 (scores_ld a multiple of 4, base 16-byte aligned)
+ *   idx     [M, k] int32 out
+ *   count   [M] int32 out (number of valid indices per row) or NULL
+ *   kth     [M] fp32 out (the smallest selected score per row; -inf for an empty row) or NULL
+ */
+size_t janus_topk_workspace_size(int M, int64_t n_keys, int k);
+int janus_topk(const float* scores, int64_t scores_ld, int M, int64_t n_keys,
+               int64_t q_pos0, int causal, int k,
+               int32_t* idx, int32_t* count, float* kth,
+               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Page demand - union of the selections (Sec. 2.2), best-effort read packing into maximal runs of physically
+ * adjacent pages (Sec. 4.3) and the corrective-read set "exact minus predicted" (Sec. 4.2).
+ *
+ *   A      = { page_table[s / page_size] : s in idx, 0 <= s < demand_limit }      (history tokens only: demand_limit = L)
+ *   bitmap = A as n_phys_pages bits (bit p of word p/32), fully overwritten
+ *   pages  = A ascending;  runs = maximal (start, len) with start..start+len-1 in A, ascending
+ *   miss   = A minus the set in predicted_bitmap, ascending;  miss_runs = its maximal runs
+ *
+ *   idx               [n_rows, k] int32, any block of selections (-1 ignored)
+ *   page_table        [n_logical_pages] int32 logical -> physical page id
+ *   predicted_bitmap  NULL (then miss = A), or the `bitmap` output of an earlier call on the predicted selection
+ *   pages, runs       out, room for `capacity` pages / `capacity` (start,len) pairs; counts in *n_pages, *n_runs (device)
+ *   miss_pages, n_miss, miss_runs, n_miss_runs   out, all four given or all four NULL
+ *
+ * If a list would exceed `capacity`, only its first `capacity` entries are written, the count still holds the
+ * true total and *dev_status becomes JANUS_DEV_CAPACITY_EXCEEDED.  Out-of-range tokens or page ids are skipped
+ * with JANUS_DEV_INDEX_OUT_OF_RANGE.  Results are bit-exact and independent of launch geometry.
+ */
+size_t janus_page_demand_workspace_size(int64_t n_rows, int k, int64_t n_phys_pages);
+int janus_page_demand(const int32_t* idx, int64_t n_rows, int k,
+                      int64_t demand_limit, int page_size,
+                      const int32_t* page_table, int64_t n_logical_pages, int64_t n_phys_pages,
+                      const uint32_t* predicted_bitmap,
+                      uint32_t* bitmap,
+                      int32_t* pages, int32_t* n_pages,
+                      int32_t* runs, int32_t* n_runs,
+                      int32_t* miss_pages, int32_t* n_miss,
+                      int32_t* miss_runs, int32_t* n_miss_runs,
+                      int64_t capacity,
+                      void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * Sparse attention over the selected rows only (Sec. 2.2, "core attention"):
+ *
+ *     out[t, h, :] = sum_{s in idx[t]} softmax_s( softmax_scale * < q[t, h, :d_qk], K_s[:d_qk] > ) * V_s[:d_v]
+ *
+ * with an fp32 online softmax.  Token s lives at element offset
+ *     page_table[s / page_size] * page_stride + (s % page_size) * tok_stride + h_kv * head_stride
+ * of k_pool (keys, d_qk values) and v_pool (values, d_v values); query head h reads kv head h * n_kv_heads / H_q.
+ * v_pool may alias k_pool (latent layout: the value is the first d_v dims of the key row).
+ *
+ *   q     [M, H_q, d_qk] bf16, dense
+ *   idx   [M, k] int32, -1 padded (any position); duplicates are attended twice
+ *   out   [M, H_q, d_v] bf16 out (round-to-nearest-even); an empty selection gives zeros
+ *   lse   [M, H_q] fp32 out, log-sum-exp of the scaled logits (-inf for an empty selection), or NULL
+ *
+ * d_qk and d_v multiples of 8, d_qk <= 576, d_v <= 512, H_q a multiple of n_kv_heads; strides (in elements)
+ * multiples of 8.  The tensor-core kernel serves the latent shape (n_kv_heads = 1, H_q = 128, d_qk = 576, d_v = 512).
+ */
+size_t janus_sparse_attn_prefill_workspace_size(int M, int H_q, int d_qk, int d_v, int k);
+int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk,
+                              const void* k_pool, const void* v_pool,
+                              int64_t page_stride, int64_t tok_stride, int64_t head_stride,
+                              int n_kv_heads, int d_v,
+                              const int32_t* idx, int k,
+                              int page_size, const int32_t* page_table, int64_t n_logical_pages,
+                              float softmax_scale,
+                              void* out, float* lse,
+                              void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JANUS_H_ */

@@ -1,0 +1,229 @@
+"""ctypes binding of libjanus.so: same names as the C entry points, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch provides device memory and the stream, nothing else); every
+step runs in the library's kernels.  There is no CPU fallback: if the library is missing or the call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import torch
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libjanus.so")
+
+JANUS_OK = 0
+ERR_NAMES = {1: "JANUS_ERR_INVALID_ARG", 2: "JANUS_ERR_UNSUPPORTED", 3: "JANUS_ERR_WORKSPACE_TOO_SMALL", 4: "JANUS_ERR_CUDA"}
+DEV_NAMES = {101: "JANUS_DEV_INDEX_OUT_OF_RANGE", 102: "JANUS_DEV_CAPACITY_EXCEEDED", 103: "JANUS_DEV_WAIT_TIMEOUT"}
+DTYPE_BF16, DTYPE_FP8_E4M3 = 0, 1
+
+# every symbol include/janus.h declares
+EXPORTS = [
+    "janus_version", "janus_last_cuda_error",
+    "janus_indexer_scores_workspace_size", "janus_indexer_scores",
+    "janus_topk_workspace_size", "janus_topk",
+    "janus_page_demand_workspace_size", "janus_page_demand",
+    "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
+]
+
+
+class JanusError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libjanus.so (built in-tree by paper_2609_36938_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise JanusError(f"{LIB_PATH} not found: build it first (python -m paper_2609_36938_b200.build); there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    c_i, c_i64, c_p, c_f, c_sz = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
+    lib.janus_version.restype = c_i
+    lib.janus_last_cuda_error.restype = c_i
+    lib.janus_indexer_scores_workspace_size.restype = c_sz
+    lib.janus_indexer_scores_workspace_size.argtypes = [c_i, c_i, c_i, c_i64, c_i]
+    lib.janus_indexer_scores.restype = c_i
+    lib.janus_indexer_scores.argtypes = [c_p, c_i64, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_i64, c_i64, c_i, c_i,
+                                         c_p, c_i64, c_p, c_sz, c_p, c_p]
+    lib.janus_topk_workspace_size.restype = c_sz
+    lib.janus_topk_workspace_size.argtypes = [c_i, c_i64, c_i]
+    lib.janus_topk.restype = c_i
+    lib.janus_topk.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p, c_p]
+    lib.janus_page_demand_workspace_size.restype = c_sz
+    lib.janus_page_demand_workspace_size.argtypes = [c_i64, c_i, c_i64]
+    lib.janus_page_demand.restype = c_i
+    lib.janus_page_demand.argtypes = [c_p, c_i64, c_i, c_i64, c_i, c_p, c_i64, c_i64, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p,
+                                      c_i64, c_p, c_sz, c_p, c_p]
+    lib.janus_sparse_attn_prefill_workspace_size.restype = c_sz
+    lib.janus_sparse_attn_prefill_workspace_size.argtypes = [c_i, c_i, c_i, c_i, c_i]
+    lib.janus_sparse_attn_prefill.restype = c_i
+    lib.janus_sparse_attn_prefill.argtypes = [c_p, c_i, c_i, c_i, c_p, c_p, c_i64, c_i64, c_i64, c_i, c_i, c_p, c_i, c_i, c_p, c_i64,
+                                              c_f, c_p, c_p, c_p, c_sz, c_p, c_p]
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != JANUS_OK:
+        extra = f" (cudaError {load().janus_last_cuda_error()})" if rc == 4 else ""
+        raise JanusError(f"{what} failed: {ERR_NAMES.get(rc, rc)}{extra}")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise JanusError("expected a CUDA tensor (the library takes device pointers)")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+_status: Dict[int, torch.Tensor] = {}
+
+
+def dev_status_tensor() -> torch.Tensor:
+    """The device status word the binding passes to every call on the current device."""
+    d = torch.cuda.current_device()
+    if d not in _status:
+        _status[d] = torch.zeros(1, dtype=torch.int32, device=f"cuda:{d}")
+    return _status[d]
+
+
+def check_dev_status(reset: bool = True) -> None:
+    """Synchronises and raises if a kernel reported a device-side condition."""
+    st = dev_status_tensor()
+    v = int(st.item())
+    if reset and v != 0:
+        st.zero_()
+    if v != 0:
+        raise JanusError(f"device status {DEV_NAMES.get(v, v)}")
+
+
+def janus_version() -> int:
+    return int(load().janus_version())
+
+
+def _idx_dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype in (torch.uint8, torch.float8_e4m3fn):
+        return DTYPE_FP8_E4M3
+    raise JanusError(f"indexer operands must be bfloat16 or E4M3 bytes, got {t.dtype}")
+
+
+def janus_indexer_scores(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, *, q_scale: Optional[torch.Tensor] = None,
+                         k_scale: Optional[torch.Tensor] = None, row_bias: Optional[torch.Tensor] = None,
+                         col_bias: Optional[torch.Tensor] = None, q_pos0: int = 0, causal: bool = True,
+                         scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """scores[t,s] = sum_h w[t,h] relu(<q_idx[t,h], k_idx[s]>) (+ row_bias[t] col_bias[s]); -inf where masked.
+    q_idx [M,H,D], k_idx [n_keys,D] (bf16 or E4M3 bytes), w [M,H] fp32.  Returns [M, ld] fp32, ld >= n_keys."""
+    lib = load()
+    M, H, D = q_idx.shape
+    n_keys = k_idx.shape[0]
+    dtype = _idx_dtype_code(q_idx)
+    if _idx_dtype_code(k_idx) != dtype:
+        raise JanusError("q_idx and k_idx must share a dtype")
+    if scores is None:
+        ld = (n_keys + 31) // 32 * 32
+        scores = torch.empty((M, ld), dtype=torch.float32, device=q_idx.device)
+    qs_stride = 0
+    if q_scale is not None and q_scale.dim() == 2:
+        qs_stride = H
+    rc = lib.janus_indexer_scores(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride,
+                                  _ptr(k_scale), _ptr(row_bias), _ptr(col_bias), M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype,
+                                  _ptr(scores), scores.stride(0), None, 0, _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_indexer_scores")
+    return scores
+
+
+def janus_topk(scores: torch.Tensor, n_keys: int, k: int, *, q_pos0: int = 0, causal: bool = True, want_count: bool = True,
+               want_kth: bool = True):
+    """Per-row top-k over the visible prefix.  Returns (idx [M,k] int32 with -1 padding, count [M] | None, kth [M] | None)."""
+    lib = load()
+    M = scores.shape[0]
+    idx = torch.empty((M, k), dtype=torch.int32, device=scores.device)
+    count = torch.empty((M,), dtype=torch.int32, device=scores.device) if want_count else None
+    kth = torch.empty((M,), dtype=torch.float32, device=scores.device) if want_kth else None
+    rc = lib.janus_topk(_ptr(scores), scores.stride(0), M, int(n_keys), int(q_pos0), int(bool(causal)), int(k), _ptr(idx), _ptr(count),
+                        _ptr(kth), None, 0, _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_topk")
+    return idx, count, kth
+
+
+def janus_page_demand(idx: torch.Tensor, *, demand_limit: int, page_size: int, page_table: torch.Tensor, n_phys_pages: int,
+                      predicted_bitmap: Optional[torch.Tensor] = None, capacity: Optional[int] = None, want_miss: bool = True):
+    """Union of selected history tokens as a physical-page bitmap, ascending page list, maximal runs and the miss set
+    against ``predicted_bitmap``.  Returns a dict of device tensors; the counts stay on the device (no host sync)."""
+    lib = load()
+    dev = idx.device
+    n_rows, k = idx.shape
+    cap = int(capacity) if capacity is not None else int(n_phys_pages)
+    n_words = (n_phys_pages + 31) // 32
+    out = {
+        "bitmap": torch.empty((n_words,), dtype=torch.int32, device=dev),
+        "pages": torch.empty((max(cap, 1),), dtype=torch.int32, device=dev),
+        "runs": torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev),
+        "counts": torch.zeros((4,), dtype=torch.int32, device=dev),   # n_pages, n_runs, n_miss, n_miss_runs
+    }
+    cp = out["counts"].data_ptr()
+    miss_args = [None, None, None, None]
+    if want_miss:
+        out["miss_pages"] = torch.empty((max(cap, 1),), dtype=torch.int32, device=dev)
+        out["miss_runs"] = torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev)
+        miss_args = [_ptr(out["miss_pages"]), cp + 8, _ptr(out["miss_runs"]), cp + 12]
+    rc = lib.janus_page_demand(_ptr(idx), n_rows, k, int(demand_limit), int(page_size), _ptr(page_table), page_table.numel(),
+                               int(n_phys_pages), _ptr(predicted_bitmap), _ptr(out["bitmap"]), _ptr(out["pages"]), cp,
+                               _ptr(out["runs"]), cp + 4, *miss_args, cap, None, 0, _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_page_demand")
+    return out
+
+
+def janus_sparse_attn_prefill(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, idx: torch.Tensor, *,
+                              page_table: torch.Tensor, page_size: int, softmax_scale: float, d_v: int,
+                              want_lse: bool = True, out: Optional[torch.Tensor] = None):
+    """Attention of each new token over its selected rows only.  q [M,H_q,d_qk] bf16; pools
+    [n_phys_pages, page_size, n_kv_heads, d] bf16 (v_pool may be k_pool itself: value = first d_v dims of the key row);
+    idx [M,k] int32.  Returns (out [M,H_q,d_v] bf16, lse [M,H_q] fp32 | None)."""
+    lib = load()
+    M, H_q, d_qk = q.shape
+    n_kv = k_pool.shape[2]
+    if out is None:
+        out = torch.empty((M, H_q, d_v), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((M, H_q), dtype=torch.float32, device=q.device) if want_lse else None
+    if v_pool.data_ptr() != k_pool.data_ptr() and v_pool.stride() != k_pool.stride():
+        raise JanusError("k_pool and v_pool must share strides")
+    rc = lib.janus_sparse_attn_prefill(_ptr(q), M, H_q, d_qk, _ptr(k_pool), _ptr(v_pool), k_pool.stride(0), k_pool.stride(1),
+                                       k_pool.stride(2), n_kv, int(d_v), _ptr(idx), idx.shape[1], int(page_size), _ptr(page_table),
+                                       page_table.numel(), float(softmax_scale), _ptr(out), _ptr(lse), None, 0,
+                                       _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_sparse_attn_prefill")
+    return out, lse
+
+
+# ---- helpers to move generator output (bit patterns) onto the device -------------------------------------------
+def to_device(x, kind: str, device="cuda") -> Optional[torch.Tensor]:
+    """numpy array -> CUDA tensor.  kind: "bf16" (uint16 bit patterns), "fp8" (uint8 codes), "f32", "i32"."""
+    import numpy as np
+
+    if x is None:
+        return None
+    if kind == "bf16":
+        return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).view(torch.bfloat16).to(device)
+    if kind == "fp8":
+        return torch.from_numpy(np.ascontiguousarray(x)).to(device)
+    if kind == "f32":
+        return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
+    if kind == "i32":
+        return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(device)
+    raise ValueError(kind)

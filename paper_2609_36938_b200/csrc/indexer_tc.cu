@@ -1,0 +1,351 @@
+// Tensor-core indexer (Eq. 1, Sec. 2.2, scoring part) for sm_100a:
+//     scores[t,s] = k_scale[s] * sum_h (w[t,h]*q_scale[h]) * relu(<q[t,h,:], k[s,:]>) + row_bias[t]*col_bias[s]
+//
+// Mapping.  The dense contraction is K . Q^T with a reduction depth of only D_I, followed by a ReLU and a
+// weighted sum over heads for every accumulator.  Keys go on the MMA M axis (128 keys -> the 128 TMEM lanes)
+// and (token, head) pairs on the N axis (256 TMEM columns = 256/H_I tokens x H_I heads), so that after a
+// tcgen05.ld every epilogue thread owns one key, holds all heads of a token in its own registers, and reduces
+// over heads with no cross-lane traffic; a warp's 32 keys are 32 consecutive floats of one score row.
+//
+// One CTA keeps NQ query sub-tiles (NQ*256 (token,head) rows, 128 KB) stationary in shared memory and streams
+// 128-key tiles past them through a TMA ring; each key tile feeds NQ MMAs (128 x 256 x D_I), whose fp32
+// accumulators alternate between the two 256-column halves of tensor memory, so the epilogue of one
+// overlaps the MMA of the next.  Warp roles: warp 0 issues TMA, warp 1 issues MMA (one thread each) and owns
+// the TMEM allocation, warps 2-9 are two epilogue groups (one per TMEM half).
+// Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT and winds down normally.
+#include "janus_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace janus {
+
+using namespace ptx;
+
+constexpr int TC_KEYS = 128;        // keys per tile = MMA M
+constexpr int TC_N = 256;           // (token, head) rows per MMA = MMA N
+constexpr int TC_THREADS = 320;     // 1 TMA warp + 1 MMA warp + 8 epilogue warps
+constexpr int TC_SMEM_BUDGET = 227 * 1024;
+constexpr int TC_MAX_STAGES = 6;
+
+struct TcParams {
+    const float* w;
+    const float* q_scale;
+    int64_t q_scale_stride_tok;
+    const float* k_scale;
+    const float* row_bias;
+    const float* col_bias;
+    float* scores;
+    int64_t ld;
+    int64_t n_keys;
+    int64_t q_pos0;
+    int M, H, causal;
+    int n_tiles;          // ceil(n_keys / 128)
+    int tiles_per_cta;    // key tiles per CTA (grid.x chunks)
+    int nq;               // query sub-tiles per CTA
+    int atoms;            // 128-byte swizzle atoms per row (row bytes / 128)
+    int stages;           // key ring depth
+    int32_t* dev_status;
+};
+
+struct TcBarriers {
+    uint64_t q_full;
+    uint64_t k_full[TC_MAX_STAGES];
+    uint64_t k_empty[TC_MAX_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    int aborted;
+};
+
+// One 32-column chunk of accumulators: ReLU, weight, reduce over heads; a token's sum is complete every H columns.
+template <int H, class Store>
+__device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const float* __restrict__ wchunk, int col0, float& acc, Store&& store) {
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+        const float4 wv = *reinterpret_cast<const float4*>(wchunk + 4 * i4);
+        const float wl[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = 4 * i4 + j;
+            acc = fmaf(wl[j], fmaxf(__uint_as_float(r[i]), 0.f), acc);
+            if (((col0 + i + 1) % H) == 0) {
+                store((col0 + i) / H, acc);
+                acc = 0.f;
+            }
+        }
+    }
+}
+
+template <int H, bool FP8>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int TPS = TC_N / H;                      // tokens per query sub-tile
+    const int atoms = p.atoms, nq = p.nq, stages = p.stages;
+    const int q_sub_bytes = atoms * TC_N * 128;        // one query sub-tile
+    const int k_stage_bytes = atoms * TC_KEYS * 128;   // one key tile
+    unsigned char* q_smem = smem;
+    unsigned char* k_smem = smem + nq * q_sub_bytes;
+    float* ws = reinterpret_cast<float*>(k_smem + stages * k_stage_bytes);   // [nq*256] w * q_scale, column order
+    float* rbs = ws + nq * TC_N;                                             // [nq*TPS] row_bias of this CTA's tokens
+    TcBarriers* bars = reinterpret_cast<TcBarriers*>(rbs + nq * TPS);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tpc = nq * TPS;                                   // tokens per CTA
+    const int t0 = blockIdx.y * tpc;
+    const int t_hi = min(p.M, t0 + tpc) - 1;                    // last real token of this CTA
+    const int tile_begin = blockIdx.x * p.tiles_per_cta;
+    const int tile_end = min(p.n_tiles, tile_begin + p.tiles_per_cta);
+    // key tiles with at least one visible (token, key) pair come first
+    int vis_end = tile_end;
+    if (p.causal) {
+        const int64_t last_visible_tile = (p.q_pos0 + t_hi) / TC_KEYS;
+        vis_end = last_visible_tile + 1 < tile_end ? static_cast<int>(last_visible_tile + 1) : tile_end;
+        if (vis_end < tile_begin) vis_end = tile_begin;
+    }
+    const int n_vis = vis_end - tile_begin;
+
+    if ((smem_u32(smem) & 1023u) != 0u) {   // swizzled tiles need 1024-byte alignment
+        if (threadIdx.x == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+        return;
+    }
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->q_full), 1);
+        for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->tmem_full[s]), 1); mbar_init(smem_u32(&bars->tmem_empty[s]), 4); }
+        bars->aborted = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_q);
+        prefetch_tensormap(&tmap_k);
+    }
+    if (warp == 1 && n_vis > 0) {
+        tmem_alloc(smem_u32(&bars->tmem_base), 512);
+        tmem_relinquish();
+    }
+    // per-column weights (w * q_scale) and per-token bias factors of this CTA
+    for (int n = threadIdx.x; n < nq * TC_N; n += TC_THREADS) {
+        const int t = t0 + n / H, h = n % H;
+        float v = 0.f;
+        if (t < p.M) {
+            v = p.w[static_cast<int64_t>(t) * H + h];
+            if (FP8) v *= p.q_scale[static_cast<int64_t>(t) * p.q_scale_stride_tok + h];
+        }
+        ws[n] = v;
+    }
+    for (int n = threadIdx.x; n < tpc; n += TC_THREADS) rbs[n] = (p.row_bias != nullptr && t0 + n < p.M) ? p.row_bias[t0 + n] : 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+    volatile int* aborted = &bars->aborted;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && n_vis > 0) {
+            const int atom_elems = FP8 ? 128 : 64;
+            const uint32_t qf = smem_u32(&bars->q_full);
+            mbar_expect_tx(qf, static_cast<uint32_t>(nq * q_sub_bytes));
+            for (int j = 0; j < nq; ++j)
+                for (int a = 0; a < atoms; ++a)
+                    tma_load_2d(smem_u32(q_smem + j * q_sub_bytes + a * TC_N * 128), &tmap_q, a * atom_elems, (t0 + j * TPS) * H, qf);
+            int issued = 0;
+            for (int it = 0; it < n_vis; ++it) {
+                const int s = it % stages;
+                const uint32_t ph = static_cast<uint32_t>(it / stages) & 1u;
+                if (!mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u) || *aborted) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); break; }
+                const uint32_t kf = smem_u32(&bars->k_full[s]);
+                mbar_expect_tx(kf, static_cast<uint32_t>(k_stage_bytes));
+                for (int a = 0; a < atoms; ++a)
+                    tma_load_2d(smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128), &tmap_k, a * atom_elems, (tile_begin + it) * TC_KEYS, kf);
+                issued = it + 1;
+            }
+            if (*aborted) {   // let the copies already in flight land before the CTA leaves
+                mbar_wait(qf, 0);
+                for (int it = max(0, issued - stages); it < issued; ++it)
+                    mbar_wait(smem_u32(&bars->k_full[it % stages]), static_cast<uint32_t>(it / stages) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && n_vis > 0) {
+            constexpr uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, TC_N);
+            bool ok = mbar_wait(smem_u32(&bars->q_full), 0);
+            uint32_t cnt = 0;
+            for (int it = 0; it < n_vis && ok; ++it) {
+                const int s = it % stages;
+                const uint32_t ph = static_cast<uint32_t>(it / stages) & 1u;
+                ok = mbar_wait(smem_u32(&bars->k_full[s]), ph) && !*aborted;
+                if (!ok) break;
+                tc_fence_after();
+                for (int j = 0; j < nq; ++j, ++cnt) {
+                    const uint32_t slot = cnt & 1u, use = cnt >> 1;
+                    ok = mbar_wait(smem_u32(&bars->tmem_empty[slot]), (use & 1u) ^ 1u) && !*aborted;
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + slot * TC_N;
+                    uint32_t acc = 0;
+                    for (int a = 0; a < atoms; ++a) {
+                        const uint32_t ka = smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128);
+                        const uint32_t qa = smem_u32(q_smem + j * q_sub_bytes + a * TC_N * 128);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per instruction (16 bf16 or 32 e4m3)
+                            umma<FP8>(d_tmem, umma_desc_sw128(ka + ks * 32), umma_desc_sw128(qa + ks * 32), idesc, acc);
+                            acc = 1;
+                        }
+                    }
+                    umma_commit(smem_u32(&bars->tmem_full[slot]));
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&bars->k_empty[s]));
+            }
+            if (!ok) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: warps 2..9
+        const int e = (warp - 2) >> 2;          // epilogue group = TMEM half it drains
+        const int quad = warp & 3;              // TMEM lanes 32*quad .. 32*quad+31
+        const float neg_inf = __int_as_float(0xff800000);
+        bool ok = true;
+        for (int it = 0; it < n_vis && ok; ++it) {
+            const int64_t s = static_cast<int64_t>(tile_begin + it) * TC_KEYS + quad * 32 + lane;
+            const bool key_ok = s < p.n_keys;
+            const float kscale = (FP8 && key_ok) ? p.k_scale[s] : 1.f;
+            const float cb = (p.col_bias != nullptr && key_ok) ? p.col_bias[s] : 0.f;
+            for (int j = e; j < nq; j += 2) {
+                const uint32_t use = static_cast<uint32_t>(it * nq + j) >> 1;
+                ok = mbar_wait(smem_u32(&bars->tmem_full[e]), use & 1u) && !*aborted;
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + e * TC_N;
+                const int tsub0 = t0 + j * TPS;
+                float acc = 0.f;
+                auto store = [&](int tt, float v) {
+                    const int t = tsub0 + tt;
+                    if (t < p.M && key_ok) {
+                        float out = v * kscale;
+                        out = fmaf(rbs[j * TPS + tt], cb, out);
+                        if (p.causal && s > p.q_pos0 + t) out = neg_inf;
+                        p.scores[static_cast<int64_t>(t) * p.ld + s] = out;
+                    }
+                };
+#pragma unroll
+                for (int c = 0; c < TC_N / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32_wait(taddr + c * 32, r);
+                    reduce_chunk<H>(r, ws + j * TC_N + c * 32, c * 32, acc, store);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[e]));
+            }
+        }
+        if (!ok && lane == 0) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }
+        // key tiles no token of this CTA may see: -inf
+        for (int tile = vis_end + e; tile < tile_end; tile += 2) {
+            const int64_t s = static_cast<int64_t>(tile) * TC_KEYS + quad * 32 + lane;
+            if (s < p.n_keys)
+                for (int t = t0; t <= t_hi; ++t) p.scores[static_cast<int64_t>(t) * p.ld + s] = neg_inf;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1 && n_vis > 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------
+PFN_encodeTiled get_encode_tiled() {
+    static PFN_encodeTiled fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_encodeTiled>(p);
+    }
+    return fn;
+}
+
+bool make_tmap_2d_sw128(CUtensorMap* map, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t row_pitch_bytes,
+                        uint32_t box_rows, uint32_t box_cols) {
+    PFN_encodeTiled enc = get_encode_tiled();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {row_pitch_bytes};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    return enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_tok, int64_t /*k_stride_tok*/, int dtype) {
+    if (!(H == 4 || H == 8 || H == 16 || H == 32 || H == 64)) return false;
+    const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
+    if (row_bytes != 128 && row_bytes != 256) return false;
+    if (q_stride_tok != static_cast<int64_t>(H) * D) return false;
+    if (static_cast<int64_t>(M) * H >= (int64_t(1) << 31) || n_keys >= (int64_t(1) << 31) - 256) return false;
+    return true;
+}
+
+template <int H, bool FP8>
+static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    indexer_tc_kernel<H, FP8><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
+
+int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok, const float* w, const float* q_scale,
+                      int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int M, int H,
+                      int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype, float* scores, int64_t ld, int32_t* dev_status,
+                      cudaStream_t stream) {
+    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3;
+    const int esz = fp8 ? 1 : 2;
+    TcParams p;
+    p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
+    p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = ld; p.n_keys = n_keys; p.q_pos0 = q_pos0;
+    p.M = M; p.H = H; p.causal = causal; p.dev_status = dev_status;
+    p.atoms = D * esz / 128;
+    p.nq = p.atoms == 1 ? 4 : 2;
+    const int tps = TC_N / H;
+    while (p.nq > 2 && static_cast<int64_t>(p.nq / 2) * tps >= M) p.nq /= 2;   // small M: do not load empty sub-tiles
+    const int q_bytes = p.nq * p.atoms * TC_N * 128;
+    const int k_stage = p.atoms * TC_KEYS * 128;
+    const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + p.nq * tps) + static_cast<int>(sizeof(TcBarriers)) + 16;
+    p.stages = (TC_SMEM_BUDGET - q_bytes - tail) / k_stage;
+    if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
+    if (p.stages < 2) return JANUS_ERR_UNSUPPORTED;
+    const size_t smem = static_cast<size_t>(q_bytes) + static_cast<size_t>(p.stages) * k_stage + tail;
+    p.n_tiles = static_cast<int>((n_keys + TC_KEYS - 1) / TC_KEYS);
+    const int tpc = p.nq * tps;
+    const int n_groups = (M + tpc - 1) / tpc;
+    int64_t per = (static_cast<int64_t>(p.n_tiles) * n_groups + 148 * 4 - 1) / (148 * 4);
+    if (per < 2) per = 2;
+    if (per > 64) per = 64;
+    p.tiles_per_cta = static_cast<int>(per);
+    dim3 grid((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, n_groups);
+    if (grid.y > 65535) return JANUS_ERR_UNSUPPORTED;
+
+    CUtensorMap tq, tk;
+    const uint32_t box_cols = fp8 ? 128 : 64;
+    if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(M) * H, D, static_cast<uint64_t>(D) * esz, TC_N, box_cols)) return JANUS_ERR_CUDA;
+    if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(n_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols))
+        return JANUS_ERR_CUDA;
+
+#define JANUS_TC_CASE(HH)                                                             \
+    case HH:                                                                          \
+        return fp8 ? launch_tc<HH, true>(tq, tk, p, grid, smem, stream) : launch_tc<HH, false>(tq, tk, p, grid, smem, stream);
+    switch (H) {
+        JANUS_TC_CASE(4)
+        JANUS_TC_CASE(8)
+        JANUS_TC_CASE(16)
+        JANUS_TC_CASE(32)
+        JANUS_TC_CASE(64)
+    }
+#undef JANUS_TC_CASE
+    return JANUS_ERR_UNSUPPORTED;
+}
+
+}  // namespace janus

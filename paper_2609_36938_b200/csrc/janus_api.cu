@@ -1,0 +1,88 @@
+// Entry points that validate arguments and pick a kernel: janus_indexer_scores, janus_sparse_attn_prefill,
+// plus the version / error queries.  janus_topk and janus_page_demand live beside their kernels.
+#include <cstdlib>
+
+#include "janus_common.cuh"
+
+namespace janus {
+
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+
+int launch_indexer_generic(const void* q_idx, int64_t q_stride_tok, const void* k_idx, int64_t k_stride_tok, const float* w,
+                           const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
+                           const float* col_bias, int M, int H, int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype,
+                           float* scores, int64_t ld, cudaStream_t stream);
+bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_tok, int64_t k_stride_tok, int dtype);
+int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok, const float* w, const float* q_scale,
+                      int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int M, int H,
+                      int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype, float* scores, int64_t ld, int32_t* dev_status,
+                      cudaStream_t stream);
+
+int launch_sparse_attn_generic(const void* q, int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
+                               int64_t tok_stride, int64_t head_stride, int n_kv_heads, int d_v, const int32_t* idx, int k,
+                               int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
+                               float* lse, int32_t* dev_status, cudaStream_t stream);
+
+}  // namespace janus
+
+extern "C" int janus_version(void) { return 100; }
+
+extern "C" int janus_last_cuda_error(void) { return janus::g_last_cuda_error; }
+
+extern "C" size_t janus_indexer_scores_workspace_size(int, int, int, int64_t, int) { return 0; }
+
+extern "C" int janus_indexer_scores(const void* q_idx, int64_t q_stride_tok, const void* k_idx, int64_t k_stride_tok, const float* w,
+                                    const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
+                                    const float* col_bias, int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal,
+                                    int dtype, float* scores, int64_t scores_ld, void* /*ws*/, size_t /*ws_bytes*/,
+                                    int32_t* dev_status, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (M < 0 || H_I <= 0 || D_I <= 0 || n_keys < 0 || q_pos0 < 0) return JANUS_ERR_INVALID_ARG;
+    if (dtype != JANUS_DTYPE_BF16 && dtype != JANUS_DTYPE_FP8_E4M3) return JANUS_ERR_UNSUPPORTED;
+    if ((D_I % 16) != 0) return JANUS_ERR_UNSUPPORTED;
+    if (M == 0 || n_keys == 0) return JANUS_OK;
+    const int esz = dtype == JANUS_DTYPE_BF16 ? 2 : 1;
+    if (!q_idx || !k_idx || !w || !scores) return JANUS_ERR_INVALID_ARG;
+    if (!aligned16(q_idx) || !aligned16(k_idx) || !aligned16(scores)) return JANUS_ERR_INVALID_ARG;
+    if (q_stride_tok < static_cast<int64_t>(H_I) * D_I || k_stride_tok < D_I) return JANUS_ERR_INVALID_ARG;
+    if ((q_stride_tok * esz) % 16 != 0 || (k_stride_tok * esz) % 16 != 0) return JANUS_ERR_INVALID_ARG;
+    if (scores_ld < n_keys || (scores_ld & 3) != 0) return JANUS_ERR_INVALID_ARG;
+    if ((row_bias == nullptr) != (col_bias == nullptr)) return JANUS_ERR_INVALID_ARG;
+    if (dtype == JANUS_DTYPE_FP8_E4M3) {
+        if (!q_scale || !k_scale) return JANUS_ERR_INVALID_ARG;
+        if (q_scale_stride_tok != 0 && q_scale_stride_tok != H_I) return JANUS_ERR_INVALID_ARG;
+    } else if (q_scale || k_scale) {
+        return JANUS_ERR_INVALID_ARG;
+    }
+    // debugging aid: JANUS_FORCE_GENERAL_INDEXER=1 routes every shape to the general kernel
+    const char* force_general = getenv("JANUS_FORCE_GENERAL_INDEXER");
+    if (!(force_general && force_general[0] == '1') && indexer_tc_supported(M, H_I, D_I, n_keys, q_stride_tok, k_stride_tok, dtype))
+        return launch_indexer_tc(q_idx, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias, M, H_I, D_I,
+                                 n_keys, q_pos0, causal, dtype, scores, scores_ld, dev_status, stream);
+    return launch_indexer_generic(q_idx, q_stride_tok, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias,
+                                  M, H_I, D_I, n_keys, q_pos0, causal, dtype, scores, scores_ld, stream);
+}
+
+extern "C" size_t janus_sparse_attn_prefill_workspace_size(int, int, int, int, int) { return 0; }
+
+extern "C" int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk, const void* k_pool, const void* v_pool,
+                                         int64_t page_stride, int64_t tok_stride, int64_t head_stride, int n_kv_heads, int d_v,
+                                         const int32_t* idx, int k, int page_size, const int32_t* page_table,
+                                         int64_t n_logical_pages, float softmax_scale, void* out, float* lse, void* /*ws*/,
+                                         size_t /*ws_bytes*/, int32_t* dev_status, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (M < 0 || H_q <= 0 || d_qk <= 0 || d_v <= 0 || n_kv_heads <= 0 || k < 0 || page_size <= 0 || n_logical_pages < 0)
+        return JANUS_ERR_INVALID_ARG;
+    if (H_q % n_kv_heads != 0) return JANUS_ERR_INVALID_ARG;
+    if ((d_qk % 8) != 0 || (d_v % 8) != 0 || d_qk > 576 || d_v > 512) return JANUS_ERR_UNSUPPORTED;
+    if (M == 0) return JANUS_OK;
+    if (!q || !k_pool || !v_pool || !out || !page_table || (k > 0 && !idx)) return JANUS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(out)) return JANUS_ERR_INVALID_ARG;
+    if ((page_stride % 8) != 0 || (tok_stride % 8) != 0 || (head_stride % 8) != 0) return JANUS_ERR_INVALID_ARG;
+    if (M > 2147483647 / 2) return JANUS_ERR_UNSUPPORTED;
+    return launch_sparse_attn_generic(q, M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, head_stride, n_kv_heads, d_v, idx, k,
+                                      page_size, page_table, n_logical_pages, softmax_scale, out, lse, dev_status, stream);
+}

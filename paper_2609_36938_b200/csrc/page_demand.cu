@@ -1,0 +1,183 @@
+// janus_page_demand: union of selected tokens -> physical page bitmap, ascending page list,
+// maximal runs of adjacent physical pages, and the miss set "exact minus predicted"
+// (union of selections: Sec. 2.2; corrective reads: Sec. 4.2; read packing: Sec. 4.3).
+//
+// Kernel 1 (mark) streams the index block with 16-byte loads and sets page bits.  When the bitmap
+// fits in shared memory each CTA ORs into a private copy first and only touches a global word once
+// per CTA; bits are tested before the atomic so a saturated union costs no atomics at all.
+// Kernel 2 (lists) is one CTA that turns a bitmap into ordered lists with block-wide scans.
+#include "janus_common.cuh"
+
+namespace janus {
+
+constexpr int MARK_THREADS = 256;
+constexpr int MARK_SMEM_WORDS = 8192;  // 32 KB: bitmaps up to 262144 pages stay in shared memory
+constexpr int LIST_THREADS = 1024;
+
+__device__ __forceinline__ void mark_one(int s, int64_t demand_limit, int page_size, int page_shift,
+                                         const int32_t* __restrict__ page_table, int64_t n_logical_pages,
+                                         int64_t n_phys_pages, uint32_t* bm, int32_t* dev_status) {
+    if (s < 0 || static_cast<int64_t>(s) >= demand_limit) return;
+    const int64_t lp = page_shift >= 0 ? (s >> page_shift) : (s / page_size);
+    if (lp >= n_logical_pages) { report(dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE); return; }
+    const int32_t p = __ldg(page_table + lp);
+    if (p < 0 || static_cast<int64_t>(p) >= n_phys_pages) { report(dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE); return; }
+    const uint32_t bit = 1u << (p & 31);
+    uint32_t* wp = bm + (p >> 5);
+    if ((*reinterpret_cast<volatile uint32_t*>(wp) & bit) == 0u) atomicOr(wp, bit);
+}
+
+template <bool USE_SMEM>
+__global__ void __launch_bounds__(MARK_THREADS)
+page_mark_kernel(const int32_t* __restrict__ idx, int64_t n_idx, int64_t demand_limit, int page_size, int page_shift,
+                 const int32_t* __restrict__ page_table, int64_t n_logical_pages, int64_t n_phys_pages,
+                 uint32_t* __restrict__ bitmap, int n_words, int32_t* dev_status) {
+    __shared__ uint32_t sbm[USE_SMEM ? MARK_SMEM_WORDS : 1];
+    uint32_t* bm = bitmap;
+    if (USE_SMEM) {
+        for (int i = threadIdx.x; i < n_words; i += MARK_THREADS) sbm[i] = 0u;
+        __syncthreads();
+        bm = sbm;
+    }
+    const int64_t n_vec = n_idx >> 2;  // idx is 16-byte aligned
+    const int4* idx4 = reinterpret_cast<const int4*>(idx);
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * MARK_THREADS;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * MARK_THREADS + threadIdx.x; i < n_vec; i += stride) {
+        const int4 v = __ldg(idx4 + i);
+        mark_one(v.x, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bm, dev_status);
+        mark_one(v.y, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bm, dev_status);
+        mark_one(v.z, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bm, dev_status);
+        mark_one(v.w, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bm, dev_status);
+    }
+    if (blockIdx.x == 0) {
+        for (int64_t i = (n_vec << 2) + threadIdx.x; i < n_idx; i += MARK_THREADS)
+            mark_one(idx[i], demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bm, dev_status);
+    }
+    if (USE_SMEM) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_words; i += MARK_THREADS) {
+            const uint32_t v = sbm[i];
+            if (v != 0u && (__ldcg(bitmap + i) & v) != v) atomicOr(bitmap + i, v);
+        }
+    }
+}
+
+// Turns one bitmap (optionally "a AND NOT b") into: ascending ids, maximal runs, counts.
+// Single CTA; words are consumed LIST_THREADS at a time, one word per thread.
+__device__ void bitmap_to_lists(const uint32_t* __restrict__ a, const uint32_t* __restrict__ not_b, int n_words,
+                                int64_t n_bits, int32_t* __restrict__ ids, int32_t* __restrict__ n_ids,
+                                int32_t* __restrict__ runs, int32_t* __restrict__ n_runs, int64_t capacity,
+                                int32_t* dev_status, int* scan_scratch) {
+    int id_base = 0, run_base = 0, end_base = 0;
+    auto word_at = [&](int i) -> uint32_t {
+        if (i < 0 || i >= n_words) return 0u;
+        uint32_t v = a[i];
+        if (not_b != nullptr) v &= ~not_b[i];
+        if (i == n_words - 1 && (n_bits & 31)) v &= (1u << (n_bits & 31)) - 1u;  // ignore bits past the last page
+        return v;
+    };
+    for (int base = 0; base < n_words; base += LIST_THREADS) {
+        const int i = base + threadIdx.x;
+        const uint32_t v = word_at(i);
+        const uint32_t prev_top = word_at(i - 1) >> 31;
+        const uint32_t next_bot = word_at(i + 1) & 1u;
+        const uint32_t starts = v & ~((v << 1) | prev_top);          // set, and the page below is not
+        const uint32_t ends = v & ~((v >> 1) | (next_bot << 31));    // set, and the page above is not
+        int tot_ids, tot_starts, tot_ends;
+        int o_id = block_exclusive_scan<LIST_THREADS>(__popc(v), scan_scratch, &tot_ids) + id_base;
+        int o_st = block_exclusive_scan<LIST_THREADS>(__popc(starts), scan_scratch, &tot_starts) + run_base;
+        int o_en = block_exclusive_scan<LIST_THREADS>(__popc(ends), scan_scratch, &tot_ends) + end_base;
+        uint32_t m = v;
+        while (m) {
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            if (o_id < capacity) ids[o_id] = i * 32 + b;
+            ++o_id;
+        }
+        m = starts;
+        while (m) {
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            if (o_st < capacity) runs[2 * o_st] = i * 32 + b;
+            ++o_st;
+        }
+        m = ends;
+        while (m) {  // the j-th end closes the j-th start; store end+1, converted to a length below
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            if (o_en < capacity) runs[2 * o_en + 1] = i * 32 + b + 1;
+            ++o_en;
+        }
+        id_base += tot_ids;
+        run_base += tot_starts;
+        end_base += tot_ends;
+    }
+    __syncthreads();
+    const int n_r = run_base < capacity ? run_base : static_cast<int>(capacity);
+    for (int j = threadIdx.x; j < n_r; j += LIST_THREADS) runs[2 * j + 1] -= runs[2 * j];
+    if (threadIdx.x == 0) {
+        *n_ids = id_base;
+        *n_runs = run_base;
+        if (id_base > capacity || run_base > capacity) report(dev_status, JANUS_DEV_CAPACITY_EXCEEDED);
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(LIST_THREADS)
+page_lists_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ predicted, int n_words, int64_t n_phys_pages,
+                  int32_t* pages, int32_t* n_pages, int32_t* runs, int32_t* n_runs,
+                  int32_t* miss_pages, int32_t* n_miss, int32_t* miss_runs, int32_t* n_miss_runs,
+                  int64_t capacity, int32_t* dev_status) {
+    __shared__ int scan_scratch[40];
+    bitmap_to_lists(bitmap, nullptr, n_words, n_phys_pages, pages, n_pages, runs, n_runs, capacity, dev_status, scan_scratch);
+    if (miss_pages != nullptr)
+        bitmap_to_lists(bitmap, predicted, n_words, n_phys_pages, miss_pages, n_miss, miss_runs, n_miss_runs, capacity,
+                        dev_status, scan_scratch);
+}
+
+}  // namespace janus
+
+extern "C" size_t janus_page_demand_workspace_size(int64_t, int, int64_t) { return 0; }
+
+extern "C" int janus_page_demand(const int32_t* idx, int64_t n_rows, int k, int64_t demand_limit, int page_size,
+                                 const int32_t* page_table, int64_t n_logical_pages, int64_t n_phys_pages,
+                                 const uint32_t* predicted_bitmap, uint32_t* bitmap, int32_t* pages, int32_t* n_pages,
+                                 int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss, int32_t* miss_runs,
+                                 int32_t* n_miss_runs, int64_t capacity, void* /*ws*/, size_t /*ws_bytes*/,
+                                 int32_t* dev_status, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n_rows < 0 || k < 0 || page_size <= 0 || n_logical_pages < 0 || n_phys_pages <= 0 || capacity < 0 || demand_limit < 0)
+        return JANUS_ERR_INVALID_ARG;
+    if (n_phys_pages > (int64_t(1) << 31) - 64) return JANUS_ERR_UNSUPPORTED;
+    if (!bitmap || !pages || !n_pages || !runs || !n_runs || !page_table) return JANUS_ERR_INVALID_ARG;
+    const int n_miss_ptrs = (miss_pages != nullptr) + (n_miss != nullptr) + (miss_runs != nullptr) + (n_miss_runs != nullptr);
+    if (n_miss_ptrs != 0 && n_miss_ptrs != 4) return JANUS_ERR_INVALID_ARG;
+    const int64_t n_idx = n_rows * static_cast<int64_t>(k);
+    if (n_idx > 0 && (!idx || !aligned16(idx))) return JANUS_ERR_INVALID_ARG;
+
+    const int n_words = static_cast<int>((n_phys_pages + 31) / 32);
+    JANUS_CUDA_CHECK(cudaMemsetAsync(bitmap, 0, sizeof(uint32_t) * n_words, stream));
+    if (n_idx > 0) {
+        int page_shift = -1;
+        if ((page_size & (page_size - 1)) == 0) {
+            page_shift = 0;
+            while ((1 << page_shift) < page_size) ++page_shift;
+        }
+        const int64_t n_vec = (n_idx + 3) / 4;
+        int64_t blocks = (n_vec + MARK_THREADS * 8 - 1) / (MARK_THREADS * 8);
+        if (blocks < 1) blocks = 1;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        if (n_words <= MARK_SMEM_WORDS)
+            page_mark_kernel<true><<<static_cast<unsigned>(blocks), MARK_THREADS, 0, stream>>>(
+                idx, n_idx, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bitmap, n_words, dev_status);
+        else
+            page_mark_kernel<false><<<static_cast<unsigned>(blocks), MARK_THREADS, 0, stream>>>(
+                idx, n_idx, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bitmap, n_words, dev_status);
+        JANUS_CUDA_CHECK(cudaGetLastError());
+    }
+    page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs,
+                                                     miss_pages, n_miss, miss_runs, n_miss_runs, capacity, dev_status);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}

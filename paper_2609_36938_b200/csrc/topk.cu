@@ -1,0 +1,282 @@
+// janus_topk: per-row selection of the k largest scores over the causal prefix (Eq. 1, Sec. 2.2).
+//
+// One CTA per query row.  The row (0.5-1 MB of fp32 at 128K-256K keys) is read from HBM once:
+//   1. a strided sample of the row (512 x 32-byte sectors) gives a conservative threshold whose
+//      expected rank is a little above k;
+//   2. one streaming pass with 16-byte loads keeps only the elements at or above that threshold
+//      in a shared-memory candidate buffer (warp-aggregated appends, ~1.5-3 % of the row);
+//   3. an exact selection runs on the candidates in shared memory: repeated 2048-bucket
+//      histograms over a shrinking key range (buckets are linear in the order-preserving integer
+//      key, so they spread over whatever range the scores occupy), until the k-th key is isolated.
+// If the sample misjudges the row (fewer than k candidates, or more than the buffer holds) the
+// same exact selection runs over the row in global memory instead; that path is slower, never
+// wrong.  Rows that fit the buffer skip the sampling step.
+#include "janus_common.cuh"
+
+namespace janus {
+
+constexpr int TK_THREADS = 512;
+constexpr int TK_CAP = 12288;       // candidate slots (key + index = 8 bytes each)
+constexpr int TK_BUCKETS = 2048;
+constexpr int TK_SAMPLE = 4096;     // 512 threads x 8 floats (one 32-byte sector each)
+
+struct TopkShared {
+    uint32_t cand_key[TK_CAP];
+    int32_t cand_idx[TK_CAP];
+    int hist[TK_BUCKETS];
+    int scan[40];
+    int n_cand;
+    int out_pos;
+    int eq_taken;
+    uint32_t red_lo, red_hi;
+    int sel_bucket, sel_above;
+};
+
+struct SmemSource {
+    const uint32_t* key;
+    const int32_t* idx;
+    int n;
+    __device__ __forceinline__ int size() const { return n; }
+    __device__ __forceinline__ uint32_t key_at(int i) const { return key[i]; }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return idx ? idx[i] : i; }
+};
+struct GlobalSource {
+    const float* row;
+    int n;
+    __device__ __forceinline__ int size() const { return n; }
+    __device__ __forceinline__ uint32_t key_at(int i) const { return float_to_key(__ldcg(row + i)); }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return i; }
+};
+
+// Exact `need`-th largest key of a source (1 <= need <= number of elements).
+// Returns the threshold key T and, in *n_eq_take, how many elements equal to T belong to the selection.
+// Every thread of the CTA must call it; results are uniform.
+template <class Src>
+__device__ uint32_t select_kth(const Src& src, int need, TopkShared& sh, int* n_eq_take) {
+    const int tid = threadIdx.x;
+    const int n = src.size();
+    // range of the active keys
+    uint32_t lo = 0xffffffffu, hi = 0u;
+    for (int i = tid; i < n; i += TK_THREADS) {
+        const uint32_t key = src.key_at(i);
+        lo = min(lo, key);
+        hi = max(hi, key);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+        hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+    }
+    if (tid == 0) { sh.red_lo = 0xffffffffu; sh.red_hi = 0u; }
+    __syncthreads();
+    if ((tid & 31) == 0) { atomicMin(&sh.red_lo, lo); atomicMax(&sh.red_hi, hi); }
+    __syncthreads();
+    lo = sh.red_lo;
+    hi = sh.red_hi;
+    __syncthreads();
+
+    for (int iter = 0; iter < 8 && lo < hi; ++iter) {
+        const uint32_t range = hi - lo;
+        const int bits = 32 - __clz(range);                   // range < 2^bits
+        const int shift = bits > 11 ? bits - 11 : 0;          // (range >> shift) < 2048
+        for (int i = tid; i < TK_BUCKETS; i += TK_THREADS) sh.hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += TK_THREADS) {
+            const uint32_t key = src.key_at(i);
+            if (key >= lo && key <= hi) atomicAdd(&sh.hist[(key - lo) >> shift], 1);
+        }
+        __syncthreads();
+        // walk the buckets from the top: thread t owns the 4 buckets 2047-4t .. 2044-4t
+        int c[4];
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { c[j] = sh.hist[TK_BUCKETS - 1 - (4 * tid + j)]; mine += c[j]; }
+        int total;
+        int above = block_exclusive_scan<TK_THREADS>(mine, sh.scan, &total);
+        if (above < need && need <= above + mine) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (above < need && need <= above + c[j]) { sh.sel_bucket = TK_BUCKETS - 1 - (4 * tid + j); sh.sel_above = above; }
+                above += c[j];
+            }
+        }
+        __syncthreads();
+        const uint32_t b = static_cast<uint32_t>(sh.sel_bucket);
+        need -= sh.sel_above;
+        const uint32_t new_lo = lo + (b << shift);
+        if (b < (range >> shift)) hi = new_lo + ((1u << shift) - 1u);   // the top bucket keeps hi (and cannot overflow)
+        lo = new_lo;
+        __syncthreads();
+    }
+    *n_eq_take = need;   // lo == hi: `need` of the elements equal to lo complete the selection
+    return lo;
+}
+
+// Writes the selection (all keys > T, plus n_eq of the keys == T) to out[0..k).
+template <class Src>
+__device__ void emit_selection(const Src& src, uint32_t T, int n_eq, int32_t* out, TopkShared& sh) {
+    const int n = src.size();
+    for (int i = threadIdx.x; i < n; i += TK_THREADS) {
+        const uint32_t key = src.key_at(i);
+        if (key > T) {
+            out[atomicAdd(&sh.out_pos, 1)] = src.idx_at(i);
+        } else if (key == T) {
+            if (atomicAdd(&sh.eq_taken, 1) < n_eq) out[atomicAdd(&sh.out_pos, 1)] = src.idx_at(i);
+        }
+    }
+}
+
+__device__ __forceinline__ void append_candidates(const float (&v)[4], int base_idx, int n_valid, uint32_t thr, TopkShared& sh) {
+    uint32_t key[4];
+    int pass = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        key[j] = float_to_key(v[j]);
+        pass += (j < n_valid && key[j] >= thr) ? 1 : 0;
+    }
+    // warp-aggregated reservation: one shared atomic per warp
+    const int lane = threadIdx.x & 31;
+    int incl = pass;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        int y = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    const int warp_total = __shfl_sync(0xffffffffu, incl, 31);
+    if (warp_total == 0) return;
+    int base = 0;
+    if (lane == 31) base = atomicAdd(&sh.n_cand, warp_total);
+    base = __shfl_sync(0xffffffffu, base, 31);
+    int pos = base + incl - pass;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (j < n_valid && key[j] >= thr) {
+            if (pos < TK_CAP) { sh.cand_key[pos] = key[j]; sh.cand_idx[pos] = base_idx + j; }
+            ++pos;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(TK_THREADS)
+topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int k,
+                 int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+    const int tid = threadIdx.x;
+    const int t = blockIdx.x;
+    const float* row = scores + static_cast<int64_t>(t) * ld;
+    int32_t* out = idx + static_cast<int64_t>(t) * k;
+    int64_t prefix64 = causal ? min(n_keys, q_pos0 + t + 1) : n_keys;
+    if (prefix64 < 0) prefix64 = 0;
+    const int n = static_cast<int>(prefix64);
+    const int n_sel = n < k ? n : k;
+
+    if (tid == 0) { sh.n_cand = 0; sh.out_pos = 0; sh.eq_taken = 0; }
+    __syncthreads();
+
+    if (n <= k) {  // the whole prefix is selected
+        for (int i = tid; i < k; i += TK_THREADS) out[i] = i < n ? i : -1;
+        if (kth != nullptr || count != nullptr) {
+            float mn = __int_as_float(0x7f800000);
+            for (int i = tid; i < n; i += TK_THREADS) mn = fminf(mn, __ldcg(row + i));
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+            if (tid == 0) sh.red_lo = 0xffffffffu;
+            __syncthreads();
+            if ((tid & 31) == 0) atomicMin(&sh.red_lo, float_to_key(mn));
+            __syncthreads();
+            if (tid == 0) {
+                if (count) count[t] = n;
+                if (kth) kth[t] = n > 0 ? key_to_float(sh.red_lo) : __int_as_float(0xff800000);
+            }
+        }
+        return;
+    }
+
+    uint32_t thr = 0u;  // keep everything
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    if (n > TK_CAP) {
+        // ---- sample: thread i reads 8 consecutive floats at an evenly spread, 32-byte aligned offset
+        const int n8 = n >> 3;                       // complete 8-float groups
+        const int g = static_cast<int>((static_cast<int64_t>(tid) * (n8 - 1)) / (TK_THREADS - 1));
+        const float4 a = __ldcg(row4 + 2 * g), b = __ldcg(row4 + 2 * g + 1);
+        uint32_t* skey = sh.cand_key;                // the candidate buffer is free at this point
+        skey[tid * 8 + 0] = float_to_key(a.x); skey[tid * 8 + 1] = float_to_key(a.y);
+        skey[tid * 8 + 2] = float_to_key(a.z); skey[tid * 8 + 3] = float_to_key(a.w);
+        skey[tid * 8 + 4] = float_to_key(b.x); skey[tid * 8 + 5] = float_to_key(b.y);
+        skey[tid * 8 + 6] = float_to_key(b.z); skey[tid * 8 + 7] = float_to_key(b.w);
+        __syncthreads();
+        // rank in the sample whose value sits a few standard deviations below the true k-th
+        const float expect = static_cast<float>(TK_SAMPLE) * static_cast<float>(k) / static_cast<float>(n);
+        int r = static_cast<int>(expect + 4.0f * sqrtf(expect) + 8.0f);
+        if (r < TK_SAMPLE) {
+            int dummy;
+            SmemSource s{skey, nullptr, TK_SAMPLE};
+            thr = select_kth(s, r, sh, &dummy);
+        }
+        __syncthreads();
+    }
+
+    // ---- one streaming pass: keep elements with key >= thr
+    {
+        const int n4 = n >> 2;
+        const int n4_round = (n4 + TK_THREADS - 1) / TK_THREADS * TK_THREADS;  // all lanes take part in the shuffles
+        for (int i = tid; i < n4_round; i += TK_THREADS) {
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            int n_valid = 0;
+            if (i < n4) {
+                const float4 x = __ldcs(row4 + i);
+                v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+                n_valid = 4;
+            }
+            append_candidates(v, 4 * i, n_valid, thr, sh);
+        }
+        {   // ragged tail (< 4 elements), handled by the first warp
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            int n_valid = 0;
+            if (tid == 0) {
+                n_valid = n - 4 * n4;
+                for (int j = 0; j < n_valid; ++j) v[j] = __ldcg(row + 4 * n4 + j);
+            }
+            if (tid < 32) append_candidates(v, 4 * n4, n_valid, thr, sh);
+        }
+    }
+    __syncthreads();
+    const int n_cand = sh.n_cand;
+    uint32_t T;
+    int n_eq;
+    if (n_cand >= k && n_cand <= TK_CAP) {
+        SmemSource s{sh.cand_key, sh.cand_idx, n_cand};
+        T = select_kth(s, k, sh, &n_eq);
+        emit_selection(s, T, n_eq, out, sh);
+    } else {
+        GlobalSource s{row, n};
+        T = select_kth(s, k, sh, &n_eq);
+        emit_selection(s, T, n_eq, out, sh);
+    }
+    if (tid == 0) {
+        if (count) count[t] = n_sel;
+        if (kth) kth[t] = key_to_float(T);
+    }
+}
+
+}  // namespace janus
+
+extern "C" size_t janus_topk_workspace_size(int, int64_t, int) { return 0; }
+
+extern "C" int janus_topk(const float* scores, int64_t scores_ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int k,
+                          int32_t* idx, int32_t* count, float* kth, void* /*ws*/, size_t /*ws_bytes*/,
+                          int32_t* /*dev_status*/, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (M < 0 || n_keys < 0 || k <= 0 || q_pos0 < 0 || scores_ld < n_keys) return JANUS_ERR_INVALID_ARG;
+    if (n_keys >= (int64_t(1) << 31) - 8) return JANUS_ERR_UNSUPPORTED;
+    if (M == 0) return JANUS_OK;
+    if (!idx) return JANUS_ERR_INVALID_ARG;
+    if (n_keys > 0 && (!scores || !aligned16(scores) || (scores_ld & 3) != 0)) return JANUS_ERR_INVALID_ARG;
+    const size_t smem = sizeof(TopkShared);
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    topk_rows_kernel<<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}

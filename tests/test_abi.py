@@ -1,0 +1,98 @@
+"""Host-side checks of the C boundary (no GPU needed): the library builds, loads and exports every symbol the
+header declares, and argument validation rejects bad calls before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_36938_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "janus.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(janus_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    declared = _declared_symbols()
+    assert len(declared) >= 10
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in janus.h but not exported"
+    assert sorted(binding.EXPORTS) == declared
+
+
+def test_version_and_workspace_queries(lib):
+    assert lib.janus_version() >= 100
+    assert lib.janus_indexer_scores_workspace_size(16, 64, 128, 4096, 0) == 0
+    assert lib.janus_topk_workspace_size(16, 4096, 64) == 0
+    assert lib.janus_page_demand_workspace_size(16, 64, 100) == 0
+    assert lib.janus_sparse_attn_prefill_workspace_size(16, 128, 576, 512, 64) == 0
+
+
+def test_invalid_arguments_are_rejected_on_the_host(lib):
+    INVALID, UNSUPPORTED = 1, 2
+    fake = ctypes.c_void_p(0x1000)       # aligned, never dereferenced: validation fails first
+    odd = ctypes.c_void_p(0x1004)
+    # indexer: bad dtype, D not a multiple of 16, NULL pointers, misaligned pointer, scores_ld too small, fp8 without scales
+    args = dict(q=fake, qs=64 * 128, k=fake, ks=128, w=fake, qsc=None, qss=0, ksc=None, rb=None, cb=None, M=4, H=64, D=128, n=256,
+                pos=0, causal=1, dt=0, sc=fake, ld=256)
+
+    def idx_call(**kw):
+        a = dict(args, **kw)
+        return lib.janus_indexer_scores(a["q"], a["qs"], a["k"], a["ks"], a["w"], a["qsc"], a["qss"], a["ksc"], a["rb"], a["cb"], a["M"],
+                                        a["H"], a["D"], a["n"], a["pos"], a["causal"], a["dt"], a["sc"], a["ld"], None, 0, None, None)
+
+    assert idx_call(dt=7) == UNSUPPORTED
+    assert idx_call(D=100) == UNSUPPORTED
+    assert idx_call(q=None) == INVALID
+    assert idx_call(q=odd) == INVALID
+    assert idx_call(ld=100) == INVALID
+    assert idx_call(ld=258) == INVALID
+    assert idx_call(dt=1) == INVALID                      # fp8 needs both scale arrays
+    assert idx_call(rb=fake) == INVALID                   # bias factors come in pairs
+    assert idx_call(M=-1) == INVALID
+    assert idx_call(M=0) == 0                             # nothing to do
+    # top-k
+    assert lib.janus_topk(fake, 256, 4, 256, 0, 1, 0, fake, None, None, None, 0, None, None) == INVALID      # k = 0
+    assert lib.janus_topk(fake, 100, 4, 256, 0, 1, 8, fake, None, None, None, 0, None, None) == INVALID      # ld < n_keys
+    assert lib.janus_topk(odd, 256, 4, 256, 0, 1, 8, fake, None, None, None, 0, None, None) == INVALID       # misaligned
+    assert lib.janus_topk(fake, 256, 4, 256, 0, 1, 8, None, None, None, None, 0, None, None) == INVALID      # no output
+    assert lib.janus_topk(fake, 256, 0, 256, 0, 1, 8, fake, None, None, None, 0, None, None) == 0            # M = 0
+    # page demand: page_size 0, missing outputs, partial miss group
+    def pd(page_size=64, bitmap=fake, miss=(None, None, None, None), n_phys=64):
+        return lib.janus_page_demand(fake, 4, 8, 100, page_size, fake, 4, n_phys, None, bitmap, fake, fake, fake, fake, *miss, 64,
+                                     None, 0, None, None)
+    assert pd(page_size=0) == INVALID
+    assert pd(bitmap=None) == INVALID
+    assert pd(miss=(fake, None, None, None)) == INVALID
+    assert pd(n_phys=0) == INVALID
+    # attention: head counts that do not divide, unsupported dims, misaligned strides
+    def at(H_q=8, n_kv=8, d_qk=128, d_v=128, tok_stride=1024, q=fake):
+        return lib.janus_sparse_attn_prefill(q, 4, H_q, d_qk, fake, fake, 65536, tok_stride, 128, n_kv, d_v, fake, 16, 64, fake, 4,
+                                             ctypes.c_float(1.0), fake, None, None, 0, None, None)
+    assert at(H_q=6, n_kv=4) == INVALID
+    assert at(d_qk=132) == UNSUPPORTED
+    assert at(d_v=1024) == UNSUPPORTED
+    assert at(tok_stride=1001) == INVALID
+    assert at(q=None) == INVALID
+
+
+def test_binding_refuses_host_tensors_and_missing_library(monkeypatch):
+    import torch
+
+    with pytest.raises(binding.JanusError):
+        binding._ptr(torch.zeros(4))
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libjanus.so")
+    with pytest.raises(binding.JanusError):
+        binding.load()
