@@ -9,7 +9,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libjanus.so")
-SOURCES = ["janus_api.cu", "indexer_generic.cu", "indexer_tc.cu", "topk.cu", "page_demand.cu", "sparse_attn_generic.cu"]
+SOURCES = ["janus_api.cu", "indexer_generic.cu", "indexer_tc.cu", "topk.cu", "page_demand.cu", "sparse_attn_generic.cu",
+           "sparse_attn_latent_tc.cu"]
 
 
 def _nvcc() -> str:
@@ -50,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= pr.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.check_call([_nvcc(), "-shared", "-o", LIB_PATH, *objs, "-lcudart_static", "-ldl", "-lrt", "-lpthread"])
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB_PATH, *objs, "-lcudart_static", "-ldl", "-lrt", "-lpthread"])
     return LIB_PATH
 
 

@@ -108,6 +108,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         if (threadIdx.x == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
         return;
     }
+    // an earlier CTA of this launch gave up on a wait: do not start new work on a broken pipeline
+    if (p.dev_status != nullptr && *reinterpret_cast<volatile int32_t*>(p.dev_status) == JANUS_DEV_WAIT_TIMEOUT) return;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->q_full), 1);

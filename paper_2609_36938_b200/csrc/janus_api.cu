@@ -24,6 +24,12 @@ int launch_sparse_attn_generic(const void* q, int M, int H_q, int d_qk, const vo
                                int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
                                float* lse, int32_t* dev_status, cudaStream_t stream);
 
+bool sparse_attn_latent_tc_supported(int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
+                                     int64_t tok_stride, int n_kv_heads, int d_v, int k);
+int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t page_stride, int64_t tok_stride, const int32_t* idx, int k,
+                                 int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
+                                 float* lse, int32_t* dev_status, cudaStream_t stream);
+
 }  // namespace janus
 
 extern "C" int janus_version(void) { return 100; }
@@ -83,6 +89,12 @@ extern "C" int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk
     if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(out)) return JANUS_ERR_INVALID_ARG;
     if ((page_stride % 8) != 0 || (tok_stride % 8) != 0 || (head_stride % 8) != 0) return JANUS_ERR_INVALID_ARG;
     if (M > 2147483647 / 2) return JANUS_ERR_UNSUPPORTED;
+    // debugging aid: JANUS_FORCE_GENERAL_ATTN=1 routes every shape to the general kernel
+    const char* force_general = getenv("JANUS_FORCE_GENERAL_ATTN");
+    if (!(force_general && force_general[0] == '1') &&
+        sparse_attn_latent_tc_supported(M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, n_kv_heads, d_v, k))
+        return launch_sparse_attn_latent_tc(q, M, k_pool, page_stride, tok_stride, idx, k, page_size, page_table, n_logical_pages,
+                                            softmax_scale, out, lse, dev_status, stream);
     return launch_sparse_attn_generic(q, M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, head_stride, n_kv_heads, d_v, idx, k,
                                       page_size, page_table, n_logical_pages, softmax_scale, out, lse, dev_status, stream);
 }
