@@ -57,19 +57,30 @@ struct TcBarriers {
 };
 
 // One 32-column chunk of accumulators: ReLU, weight, reduce over heads; a token's sum is complete every H columns.
+// Pairs of columns go through packed fp32 FMAs into up to four independent accumulator pairs, so the reduction is
+// neither one long dependent chain nor one instruction per element.
 template <int H, class Store>
-__device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const float* __restrict__ wchunk, int col0, float& acc, Store&& store) {
+__device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const float* __restrict__ wchunk, int col0, float2 (&acc)[4], Store&& store) {
+    constexpr int NACC = (H / 2 < 4) ? H / 2 : 4;
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
         const float4 wv = *reinterpret_cast<const float4*>(wchunk + 4 * i4);
-        const float wl[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int i = 4 * i4 + j;
-            acc = fmaf(wl[j], fmaxf(__uint_as_float(r[i]), 0.f), acc);
-            if (((col0 + i + 1) % H) == 0) {
-                store((col0 + i) / H, acc);
-                acc = 0.f;
+        for (int j = 0; j < 2; ++j) {
+            const int i = 4 * i4 + 2 * j;                      // first column of the pair inside the chunk
+            const int col = col0 + i;
+            const float2 w2 = j == 0 ? make_float2(wv.x, wv.y) : make_float2(wv.z, wv.w);
+            const float2 x2 = make_float2(fmaxf(__uint_as_float(r[i]), 0.f), fmaxf(__uint_as_float(r[i + 1]), 0.f));
+            float2& a = acc[(col / 2) % NACC];
+            a = ffma2(w2, x2, a);
+            if (((col + 2) % H) == 0) {
+                float v = 0.f;
+#pragma unroll
+                for (int q = 0; q < NACC; ++q) {
+                    v += acc[q].x + acc[q].y;
+                    acc[q] = make_float2(0.f, 0.f);
+                }
+                store(col / H, v);
             }
         }
     }
@@ -220,7 +231,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + e * TC_N;
                 const int tsub0 = t0 + j * TPS;
-                float acc = 0.f;
+                float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 auto store = [&](int tt, float v) {
                     const int t = tsub0 + tt;
                     if (t < p.M && key_ok) {
@@ -230,15 +241,25 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                         p.scores[static_cast<int64_t>(t) * p.ld + s] = out;
                     }
                 };
+                // two register buffers: the load of the next 32 columns is in flight while this one is reduced
+                uint32_t ra[32], rb[32];
+                tmem_ld32_issue(taddr, ra);
 #pragma unroll
-                for (int c = 0; c < TC_N / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32_wait(taddr + c * 32, r);
-                    reduce_chunk<H>(r, ws + j * TC_N + c * 32, c * 32, acc, store);
+                for (int c = 0; c < TC_N / 32; c += 2) {
+                    tmem_ld_wait(ra);
+                    tmem_ld32_issue(taddr + (c + 1) * 32, rb);
+                    reduce_chunk<H>(ra, ws + j * TC_N + c * 32, c * 32, acc, store);
+                    tmem_ld_wait(rb);
+                    if (c + 2 < TC_N / 32) {
+                        tmem_ld32_issue(taddr + (c + 2) * 32, ra);
+                    } else {
+                        // every column of this TMEM half is in registers: hand it back before the last reduction
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[e]));
+                    }
+                    reduce_chunk<H>(rb, ws + j * TC_N + (c + 1) * 32, (c + 1) * 32, acc, store);
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[e]));
             }
         }
         if (!ok && lane == 0) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }

@@ -188,25 +188,35 @@ sparse_attn_latent_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const L
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->k_full[j % LA_STAGES]));
         };
+        // Address resolution runs ahead of the copies so that neither the index load (HBM) nor the page-table load sits
+        // on the per-tile critical path: indices are fetched two tiles ahead, page ids one tile ahead.
+        auto load_raw = [&](int tile) -> int {
+            const int slot = tile * LA_BK + lane;
+            return (tile < n_tiles && slot < p.k) ? __ldg(my_idx + slot) : -1;
+        };
+        auto page_of = [&](int s_tok, int& within) -> int {   // returns the physical page id (or -1), issues the table load
+            within = 0;
+            if (s_tok < 0) return -1;
+            const int64_t lp = p.page_shift >= 0 ? (s_tok >> p.page_shift) : (s_tok / p.page_size);
+            within = p.page_shift >= 0 ? (s_tok & (p.page_size - 1)) : (s_tok % p.page_size);
+            if (lp >= p.n_logical_pages) { report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE); return -1; }
+            return __ldg(p.page_table + lp);
+        };
+        int within_cur, within_nxt = 0;
+        int page_cur = page_of(load_raw(0), within_cur);     // tile 0
+        int raw_nxt = load_raw(1);                            // tile 1 (translated in iteration 0)
+        int page_nxt = -1;
         for (int i = 0; i < n_tiles; ++i) {
             const int st = i % LA_STAGES;
+            const int raw_nxt2 = load_raw(i + 2);             // consumed next iteration
+            page_nxt = page_of(raw_nxt, within_nxt);          // table load issued now, consumed next iteration
             if (ok) ok = mbar_wait(smem_u32(&sh->k_empty[st]), (static_cast<uint32_t>(i / LA_STAGES) & 1u) ^ 1u) && !*aborted;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            // lane r resolves the address of row r of the tile
-            const int slot = i * LA_BK + lane;
-            int s = slot < p.k ? __ldg(my_idx + slot) : -1;
+            // lane r holds the address of row r of the tile
+            const int s = page_cur;                           // >= 0 iff the row is valid
             const unsigned char* row_ptr = reinterpret_cast<const unsigned char*>(p.pool);
-            if (s >= 0) {
-                const int64_t lp = p.page_shift >= 0 ? (s >> p.page_shift) : (s / p.page_size);
-                const int within = p.page_shift >= 0 ? (s & (p.page_size - 1)) : (s % p.page_size);
-                if (lp >= p.n_logical_pages) {
-                    report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
-                    s = -1;
-                } else {
-                    row_ptr += (static_cast<int64_t>(__ldg(p.page_table + lp)) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
-                }
-            }
+            if (s >= 0) row_ptr += (static_cast<int64_t>(page_cur) * p.page_stride + static_cast<int64_t>(within_cur) * p.tok_stride) * 2;
             const uint32_t valid_mask = __ballot_sync(0xffffffffu, s >= 0);
             if (g == 0 && lane == 0) sh->vmask[st] = valid_mask;
             const uint32_t stage_base = smem_u32(k_smem + st * LA_STAGE_BYTES);
@@ -226,6 +236,7 @@ sparse_attn_latent_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const L
                 }
             }
             cp_async_commit();
+            page_cur = page_nxt; within_cur = within_nxt; raw_nxt = raw_nxt2;
             if (i >= LA_LAG) {
                 cp_async_wait<LA_LAG>();
                 arrive_tile(i - LA_LAG);

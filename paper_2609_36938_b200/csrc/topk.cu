@@ -4,7 +4,7 @@
 //   1. a strided sample of the row (512 x 32-byte sectors) gives a conservative threshold whose
 //      expected rank is a little above k;
 //   2. one streaming pass with 16-byte loads keeps only the elements at or above that threshold
-//      in a shared-memory candidate buffer (warp-aggregated appends, ~1.5-3 % of the row);
+//      in a shared-memory candidate buffer (~1.5-3 % of the row pass the one-compare filter);
 //   3. an exact selection runs on the candidates in shared memory: repeated 2048-bucket
 //      histograms over a shrinking key range (buckets are linear in the order-preserving integer
 //      key, so they spread over whatever range the scores occupy), until the k-th key is isolated.
@@ -126,34 +126,12 @@ __device__ void emit_selection(const Src& src, uint32_t T, int n_eq, int32_t* ou
     }
 }
 
-__device__ __forceinline__ void append_candidates(const float (&v)[4], int base_idx, int n_valid, uint32_t thr, TopkShared& sh) {
-    uint32_t key[4];
-    int pass = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        key[j] = float_to_key(v[j]);
-        pass += (j < n_valid && key[j] >= thr) ? 1 : 0;
-    }
-    // warp-aggregated reservation: one shared atomic per warp
-    const int lane = threadIdx.x & 31;
-    int incl = pass;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += y;
-    }
-    const int warp_total = __shfl_sync(0xffffffffu, incl, 31);
-    if (warp_total == 0) return;
-    int base = 0;
-    if (lane == 31) base = atomicAdd(&sh.n_cand, warp_total);
-    base = __shfl_sync(0xffffffffu, base, 31);
-    int pos = base + incl - pass;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        if (j < n_valid && key[j] >= thr) {
-            if (pos < TK_CAP) { sh.cand_key[pos] = key[j]; sh.cand_idx[pos] = base_idx + j; }
-            ++pos;
-        }
+// Keeps x (at row position i) if it is at or above the streaming threshold.  The float comparison admits a superset of
+// the exact key comparison (it treats -0 and +0 alike); the exact selection afterwards works on keys.
+__device__ __forceinline__ void keep_if_candidate(float x, int i, float thr_f, TopkShared& sh) {
+    if (x >= thr_f) {
+        const int pos = atomicAdd(&sh.n_cand, 1);
+        if (pos < TK_CAP) { sh.cand_key[pos] = float_to_key(x); sh.cand_idx[pos] = i; }
     }
 }
 
@@ -217,29 +195,33 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_
         __syncthreads();
     }
 
-    // ---- one streaming pass: keep elements with key >= thr
+    // ---- one streaming pass: keep elements at or above the threshold (a few per cent of the row)
     {
+        const float thr_f = thr == 0u ? __int_as_float(0xff800000) : key_to_float(thr);
         const int n4 = n >> 2;
-        const int n4_round = (n4 + TK_THREADS - 1) / TK_THREADS * TK_THREADS;  // all lanes take part in the shuffles
-        for (int i = tid; i < n4_round; i += TK_THREADS) {
-            float v[4] = {0.f, 0.f, 0.f, 0.f};
-            int n_valid = 0;
-            if (i < n4) {
-                const float4 x = __ldcs(row4 + i);
-                v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-                n_valid = 4;
+        constexpr int UNROLL = 4;                     // 16-byte loads in flight per thread
+        int i = tid;
+        for (; i + (UNROLL - 1) * TK_THREADS < n4; i += UNROLL * TK_THREADS) {
+            float4 x[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) x[u] = __ldcs(row4 + i + u * TK_THREADS);
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int e = 4 * (i + u * TK_THREADS);
+                keep_if_candidate(x[u].x, e, thr_f, sh);
+                keep_if_candidate(x[u].y, e + 1, thr_f, sh);
+                keep_if_candidate(x[u].z, e + 2, thr_f, sh);
+                keep_if_candidate(x[u].w, e + 3, thr_f, sh);
             }
-            append_candidates(v, 4 * i, n_valid, thr, sh);
         }
-        {   // ragged tail (< 4 elements), handled by the first warp
-            float v[4] = {0.f, 0.f, 0.f, 0.f};
-            int n_valid = 0;
-            if (tid == 0) {
-                n_valid = n - 4 * n4;
-                for (int j = 0; j < n_valid; ++j) v[j] = __ldcg(row + 4 * n4 + j);
-            }
-            if (tid < 32) append_candidates(v, 4 * n4, n_valid, thr, sh);
+        for (; i < n4; i += TK_THREADS) {
+            const float4 x = __ldcs(row4 + i);
+            keep_if_candidate(x.x, 4 * i, thr_f, sh);
+            keep_if_candidate(x.y, 4 * i + 1, thr_f, sh);
+            keep_if_candidate(x.z, 4 * i + 2, thr_f, sh);
+            keep_if_candidate(x.w, 4 * i + 3, thr_f, sh);
         }
+        if (tid < n - 4 * n4) keep_if_candidate(__ldcg(row + 4 * n4 + tid), 4 * n4 + tid, thr_f, sh);   // ragged tail
     }
     __syncthreads();
     const int n_cand = sh.n_cand;
