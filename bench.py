@@ -178,7 +178,7 @@ def main():
     import torch
     import torch.distributed as dist
 
-    from paper_2609_36938_b200 import binding as B, build as _build
+    from paper_2609_36938_b200 import binding as B, build as _build, dist_utils as D
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -280,12 +280,8 @@ def main():
     B.check_dev_status()
     elapsed_ms = t_start.elapsed_time(t_end)
     per_call = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])   # [steps, 4] ms
-    if world > 1:
-        tt = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
+    value, elapsed_ms, _ = D.aggregate_throughput(float(shp.M * args.steps), elapsed_ms, device="cuda")   # max over ranks
     ms_per_step = elapsed_ms / args.steps
-    value = world * shp.M / (ms_per_step * 1e-3)
 
     # ---- end to end: every step uploads all inputs from pinned host memory and reads the results back
     e2e = None
@@ -313,12 +309,9 @@ def main():
             e2e_step()
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
-        e2e = {"value": world * shp.M / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
+        e2e_value, e2e_total_ms, _ = D.aggregate_throughput(float(shp.M * n_e2e), e0.elapsed_time(e1), device="cuda")
+        e2e_ms = e2e_total_ms / n_e2e
+        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
                "ms_per_step": e2e_ms, "inputs": "all operands (queries, keys, weights, Q, KV pool, page table) uploaded every step"}
 
     if rank != 0:

@@ -204,11 +204,11 @@ def page_demand(idx, demand_limit: int, page_size: int, page_table, predicted_pa
     Returns dict(pages=sorted(A), runs=maximal runs of A, miss=sorted(A - predicted),
     miss_runs=maximal runs of the miss set)."""
     table = np.asarray(page_table)
+    flat = np.asarray(idx).reshape(-1)
+    tokens = np.unique(flat[(flat >= 0) & (flat < demand_limit)])   # distinct selected history tokens (library sort)
     demand = set()
-    for s in np.asarray(idx).reshape(-1):
-        s = int(s)
-        if 0 <= s < demand_limit:
-            demand.add(int(table[s // page_size]))
+    for s in tokens:
+        demand.add(int(table[int(s) // page_size]))
     pages = sorted(demand)
     pred = set(int(p) for p in predicted_pages) if predicted_pages is not None else set()
     miss = sorted(demand - pred)
