@@ -91,7 +91,7 @@ extern "C" int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk
     if (M > 2147483647 / 2) return JANUS_ERR_UNSUPPORTED;
     // debugging aid: JANUS_FORCE_GENERAL_ATTN=1 routes every shape to the general kernel
     const char* force_general = getenv("JANUS_FORCE_GENERAL_ATTN");
-    if (!(force_general && force_general[0] == '1') &&
+    if (!(force_general && force_general[0] == '1') && softmax_scale > 0.f &&
         sparse_attn_latent_tc_supported(M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, n_kv_heads, d_v, k))
         return launch_sparse_attn_latent_tc(q, M, k_pool, page_stride, tok_stride, idx, k, page_size, page_table, n_logical_pages,
                                             softmax_scale, out, lse, dev_status, stream);

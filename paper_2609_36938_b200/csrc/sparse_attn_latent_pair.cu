@@ -1,0 +1,564 @@
+// Tensor-core sparse attention for the latent layout (Sec. 2.2, "core attention"): one shared KV row of 576 bf16
+// per token (keys = all 576 dims, values = the first 512), 128 query heads, selection idx[t, 0:k).
+//
+//     out[t,h,:] = sum_{s in idx[t]} softmax_s(scale * <q[t,h,:576], row_s[:576]>) * row_s[:512]
+//
+// Shape of the problem.  The heads of one token form the MMA M axis (128 heads = 128 TMEM lanes), so the fp32 output
+// accumulator, 128 lanes x 512 columns, is all of one SM's tensor memory.  One token is therefore handled by a
+// cluster of two CTAs that split the work along the *feature* axis, so that nothing is computed or fetched twice:
+//
+//   CTA 0 owns row bytes [0,512)    = dims [0,256):    value half 0, and the first 256 dims of the logit contraction;
+//   CTA 1 owns row bytes [512,1152) = dims [256,576):  value half 1, and the last 320 dims of the contraction.
+//
+// Each CTA gathers only its own bytes of every selected row, computes a partial logit tile S_c = Q_c . K_c^T
+// (128 heads x 64 keys, fp32 in TMEM), and the two partial tiles are exchanged through distributed shared memory:
+// every softmax thread (thread = head) sends its 64 partial logits into the peer's exchange buffer with asynchronous
+// remote stores that are counted on the peer's mbarrier as they land, waits for the peer's values and adds them.  Both CTAs then run the same fp32 online softmax on
+// identical sums, write P (bf16) back to TMEM over the logits, and accumulate O_c += P . V_c with V_c read MN-major
+// from the gathered rows (the value half of CTA c is the first 256 dims of the bytes it owns).
+//
+// Per CTA: queries live in tensor memory as the A operand (4 atoms of 64 dims = 128 columns; the fifth atom of
+// CTA 1, the 64 rope dims, sits in shared memory); tensor memory = O 256 | two logit buffers of 64 | Q 128 columns.
+// Keys move in half-tiles of 32 rows through a ring of three 64-key tiles.  Warp roles (15 warps):
+//   warp 0       issues the MMAs: S for tile i+1 (16 or 20 MMAs 128x64x16) before O += P.V of tile i (4 MMAs 128x256x16);
+//   warps 1-6    gather: each owns one ring slot, resolves its 32 rows through the page table (one half-tile ahead)
+//                and copies this CTA's bytes with 16-byte cp.async into the 128-byte-swizzled K-major layout;
+//   warps 7-10   exchange: as soon as a partial logit tile is complete they send it to the peer, so the transfer of
+//                tile i+1 overlaps the softmax of tile i;
+//   warps 11-14  softmax (thread = head): add the peer's partial logits, fp32 online softmax, write P (bf16) over the logits.
+// The running max only moves when a tile exceeds it by more than 2^8, so O is rescaled (in TMEM) a handful of times
+// per row.  Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT, and both CTAs of the cluster
+// still meet at the final cluster barrier.
+#include "janus_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace janus {
+
+using namespace ptx;
+
+constexpr int LP_HEADS = 128;
+constexpr int LP_DQK = 576;
+constexpr int LP_DV = 512;
+constexpr int LP_DVH = 256;
+constexpr int LP_HALF = 32;                 // rows per half-tile (gather / ring-slot granularity)
+constexpr int LP_TILE = 2 * LP_HALF;        // keys per MMA tile
+constexpr int LP_BUFS = 3;                  // 64-key tile buffers
+constexpr int LP_SLOTS = 2 * LP_BUFS;       // ring slots (half-tiles)
+constexpr int LP_GATHER_WARPS = 6;          // one per ring slot (must divide LP_SLOTS)
+constexpr int LP_ATOMS_MAX = 5;             // 64-dim atoms owned by a CTA: 4 (CTA 0) or 5 (CTA 1)
+constexpr int LP_K_ATOM_BYTES = LP_TILE * 128;                   // 8 KB
+constexpr int LP_TILE_BYTES = LP_ATOMS_MAX * LP_K_ATOM_BYTES;    // 40 KB
+constexpr int LP_XBUF_BYTES = LP_TILE * LP_HEADS * 4;            // 32 KB: partial logits from the peer, [key/4][head][4] fp32
+constexpr int LP_Q_ATOM_BYTES = LP_HEADS * 128;                  // 16 KB
+constexpr int LP_XCHG_WARP0 = 1 + LP_GATHER_WARPS;               // first exchange warp
+constexpr int LP_SMAX_WARP0 = LP_XCHG_WARP0 + 4;                 // first softmax warp
+constexpr int LP_THREADS = 32 * (LP_SMAX_WARP0 + 4);             // 15 warps
+constexpr uint32_t LP_COL_O = 0, LP_COL_S = 256, LP_COL_Q = 384;
+
+struct LpShared {
+    uint64_t q_full, qt_full;
+    uint64_t k_full[LP_BUFS], k_empty[LP_BUFS];   // per tile buffer: rows landed (2 half-tiles) / P.V of the tile done
+    uint64_t s_full[2], p_full[2];
+    uint64_t x_full[2];                           // the peer's partial logits of the tile using logit buffer b have arrived
+    uint64_t x_empty[2];                          // the PEER has read this CTA's previous partial logits out of its exchange buffer b
+    uint64_t x_sent[2];                           // this CTA's exchange warps have read logit buffer b (P may overwrite it)
+    uint32_t vmask[LP_SLOTS];
+    uint32_t tmem_base;
+    uint32_t start_abort[2];
+};
+
+struct LpParams {
+    const uint16_t* q;
+    const uint16_t* pool;
+    int64_t page_stride, tok_stride;
+    const int32_t* idx;
+    int k;
+    int page_size, page_shift;
+    const int32_t* page_table;
+    int64_t n_logical_pages;
+    float scale_log2e;        // softmax_scale * log2(e)
+    uint16_t* out;
+    float* lse;
+    int M;
+    int32_t* dev_status;
+};
+
+// Optional per-role cycle accounting for tuning (off in the product build): with -DJANUS_ATTN_PROFILE the lse output of
+// token t receives, instead of the log-sum-exp, the cycles each role of CTA 0 spent in total and inside its waits.
+#ifdef JANUS_ATTN_PROFILE
+#define LP_PROF_DECL(name) long long name = 0
+#define LP_PROF_WAIT(acc, expr) ([&] { const long long _t0 = clock64(); const bool _r = (expr); acc += clock64() - _t0; return _r; }())
+#define LP_PROF_NOW() clock64()
+#define LP_PROF_SEG(acc, t_prev) do { const long long _n = clock64(); acc += _n - t_prev; t_prev = _n; } while (0)
+#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == 0u) p.lse[static_cast<int64_t>(t) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
+#else
+#define LP_PROF_DECL(name)
+#define LP_PROF_WAIT(acc, expr) (expr)
+#define LP_PROF_NOW() 0
+#define LP_PROF_SEG(acc, t_prev) do { } while (0)
+#define LP_PROF_PUT(slot, v) do { } while (0)
+#endif
+
+__device__ __forceinline__ float lp_exp2(float x) {   // ex2.approx: 2 ulp, exp2(-inf) = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t lp_pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(LP_THREADS, 1)
+sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const LpParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char* k_smem = smem;                                              // 3 tiles x 5 atoms x [64 keys x 128 B]
+    float* xbuf = reinterpret_cast<float*>(smem + LP_BUFS * LP_TILE_BYTES);    // 2 x [64 keys][128 heads]
+    unsigned char* q4_smem = smem + LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES;   // CTA 1: query dims [512,576)
+    LpShared* sh = reinterpret_cast<LpShared*>(q4_smem + LP_Q_ATOM_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t c = cluster_ctarank();          // 0 or 1: which bytes of the rows this CTA owns
+    const uint32_t peer = c ^ 1u;
+    const int t = blockIdx.x >> 1;
+    const int n_atoms = 4 + static_cast<int>(c);
+    const int n_tiles = (p.k + LP_TILE - 1) / LP_TILE;
+    const int n_half = 2 * n_tiles;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&sh->q_full), 1);
+        mbar_init(smem_u32(&sh->qt_full), 4);
+        for (int s = 0; s < LP_BUFS; ++s) { mbar_init(smem_u32(&sh->k_full[s]), 2); mbar_init(smem_u32(&sh->k_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->s_full[b]), 1);
+            mbar_init(smem_u32(&sh->p_full[b]), 4);
+            mbar_init(smem_u32(&sh->x_full[b]), 1);
+            mbar_init(smem_u32(&sh->x_empty[b]), 4);
+            mbar_init(smem_u32(&sh->x_sent[b]), 4);
+        }
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_q);
+        // start-up agreement: if this CTA should not start (misaligned shared memory, or an earlier CTA of the launch gave
+        // up on a wait), both CTAs of the cluster must skip the work, so the flag is written to both of them
+        uint32_t flag = ((smem_u32(smem) & 1023u) != 0u) ? 1u : 0u;
+        if (p.dev_status != nullptr && *reinterpret_cast<volatile int32_t*>(p.dev_status) == JANUS_DEV_WAIT_TIMEOUT) flag = 1u;
+        sh->start_abort[c] = flag;
+        st_cluster_u32(mapa_shared(smem_u32(&sh->start_abort[c]), peer), flag);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&sh->tmem_base), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                            // barriers of both CTAs are initialised, start flags exchanged
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+    const bool start_abort = (sh->start_abort[0] | sh->start_abort[1]) != 0u;
+    if (start_abort && threadIdx.x == 0 && (smem_u32(smem) & 1023u) != 0u) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+
+    if (start_abort) {
+        // nothing to do
+    } else if (warp == 0) {
+        // ================================================================== MMA issue (whole warp runs the loop, lane 0 issues)
+        const bool leader = lane == 0;
+        const uint32_t qf = smem_u32(&sh->q_full);
+        if (leader) {
+            if (c == 1u) {
+                mbar_expect_tx(qf, LP_Q_ATOM_BYTES);
+                tma_load_2d(smem_u32(q4_smem), &tmap_q, 512, t * LP_HEADS, qf);     // rope dims [512,576) of all heads
+            } else {
+                mbar_arrive(qf);
+            }
+        }
+        constexpr uint32_t idesc_qk = umma_idesc_major(1u, LP_HEADS, LP_TILE, 0u, 0u);
+        constexpr uint32_t idesc_pv = umma_idesc_major(1u, LP_HEADS, LP_DVH, 0u, 1u);
+        LP_PROF_DECL(w_kfull); LP_PROF_DECL(w_pfull); LP_PROF_DECL(w_q);
+        const long long prof_t0 = LP_PROF_NOW();
+        bool ok = LP_PROF_WAIT(w_q, mbar_wait(qf, 0) && mbar_wait(smem_u32(&sh->qt_full), 0));
+        tc_fence_after();
+        const uint32_t q4_lo = umma_desc_lo(smem_u32(q4_smem), 16);
+        const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem), 16);
+        const uint32_t v_lo = umma_desc_lo(smem_u32(k_smem), LP_K_ATOM_BYTES);     // value half = first four owned atoms
+        auto issue_pv = [&](int j) {   // O += P_j . V_j
+            const int b = j & 1, buf = j % LP_BUFS;
+            const uint32_t vb = v_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
+            const uint32_t pa = tmem_base + LP_COL_S + b * LP_TILE;
+            if (leader) {
+#pragma unroll
+                for (int ks = 0; ks < LP_TILE / 16; ++ks)
+                    umma_bf16_ts_lohi(tmem_base + LP_COL_O, pa + ks * 8, vb + ks * (2048 >> 4), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(smem_u32(&sh->k_empty[buf]));   // tile buffer free again, and "P.V of tile j done" for the softmax warps
+            }
+        };
+        for (int i = 0; i < n_tiles && ok; ++i) {
+            const int b = i & 1, buf = i % LP_BUFS;
+            ok = LP_PROF_WAIT(w_kfull, mbar_wait(smem_u32(&sh->k_full[buf]), static_cast<uint32_t>(i / LP_BUFS) & 1u));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_s = tmem_base + LP_COL_S + b * LP_TILE;
+            const uint32_t kb = k_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
+            if (leader) {
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16_ts_lohi(d_s, tmem_base + LP_COL_Q + a * 32 + ks * 8, kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk,
+                                          (a > 0 || ks > 0) ? 1u : 0u);
+                }
+                if (c == 1u) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16_ss_lohi(d_s, q4_lo + ks * 2, kb + 4 * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk, 1u);
+                }
+                umma_commit(smem_u32(&sh->s_full[b]));
+            }
+            if (i >= 1) {
+                ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(i - 1) & 1]), static_cast<uint32_t>((i - 1) >> 1) & 1u));
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(i - 1);
+            }
+        }
+        if (ok && n_tiles > 0) {
+            ok = mbar_wait(smem_u32(&sh->p_full[(n_tiles - 1) & 1]), static_cast<uint32_t>((n_tiles - 1) >> 1) & 1u);
+            if (ok) {
+                tc_fence_after();
+                issue_pv(n_tiles - 1);
+            }
+        }
+        if (!ok && leader) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+        if (leader) { LP_PROF_PUT(0, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(1, w_kfull); LP_PROF_PUT(2, w_pfull); LP_PROF_PUT(9, w_q); }
+    } else if (warp <= LP_GATHER_WARPS) {
+        // ================================================================== gather: warp g owns ring slot g (half-tiles g, g+6, ...)
+        // A warp copies whole half-tiles (32 rows, this CTA's bytes of each), so address resolution is done once per
+        // half-tile and no two warps ever synchronise.  Because every use of a slot is made by the same warp, the slot's
+        // barrier is at most one phase ahead of it, which the parity wait relies on.
+        const int g = warp - 1;
+        const int32_t* my_idx = p.idx + static_cast<int64_t>(t) * p.k;
+        const int n_chunks = 8 * n_atoms;                      // 16-byte chunks of a row owned by this CTA (32 or 40)
+        const int64_t seg_off = 512 * static_cast<int64_t>(c); // first owned byte of a row
+        bool ok = true;
+        LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
+        const long long prof_t0 = LP_PROF_NOW();
+        auto load_raw = [&](int hi) -> int {                   // lane r owns row r of half-tile hi
+            const int slot = hi * LP_HALF + lane;
+            return (hi < n_half && slot < p.k) ? __ldg(my_idx + slot) : -1;
+        };
+        auto resolve = [&](int s_tok, bool& valid) -> const unsigned char* {   // first owned byte of the row of token s_tok
+            const unsigned char* ptr = reinterpret_cast<const unsigned char*>(p.pool) + seg_off;
+            valid = false;
+            if (s_tok >= 0) {
+                const int64_t lp = p.page_shift >= 0 ? (s_tok >> p.page_shift) : (s_tok / p.page_size);
+                const int within = p.page_shift >= 0 ? (s_tok & (p.page_size - 1)) : (s_tok % p.page_size);
+                if (lp >= p.n_logical_pages) {
+                    report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
+                } else {
+                    ptr += (static_cast<int64_t>(__ldg(p.page_table + lp)) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
+                    valid = true;
+                }
+            }
+            return ptr;
+        };
+        // rows are resolved one half-tile ahead and indices fetched two ahead, so neither load is waited for in the loop
+        bool valid_cur, valid_nxt = false;
+        const unsigned char* row_ptr = resolve(load_raw(g), valid_cur);
+        const unsigned char* row_nxt = row_ptr;
+        int raw_nxt = load_raw(g + LP_GATHER_WARPS);
+        for (int hi = g; hi < n_half; hi += LP_GATHER_WARPS) {
+            const int buf = (hi >> 1) % LP_BUFS, hf = hi & 1;
+            const bool s_ok = valid_cur;
+            const uint32_t valid_mask = __ballot_sync(0xffffffffu, s_ok);
+            // the tile buffer must have been released by the P.V three tiles back
+            ok = LP_PROF_WAIT(w_kempty, mbar_wait(smem_u32(&sh->k_empty[buf]), (static_cast<uint32_t>((hi >> 1) / LP_BUFS) & 1u) ^ 1u));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) sh->vmask[2 * buf + hf] = valid_mask;
+            const uint32_t stage_base = smem_u32(k_smem + buf * LP_TILE_BYTES + hf * LP_HALF * 128);
+            // lane l copies 16-byte chunk l (and chunk 32+l of a 640-byte segment) of every row: chunk ch of the owned bytes
+            // goes to atom ch/8, position (ch%8) ^ (r%8) inside the 128-byte row r
+            const uint32_t dst0 = stage_base + (lane >> 3) * LP_K_ATOM_BYTES + ((lane & 7) << 4);
+            const uint32_t dst1 = dst0 + 4 * LP_K_ATOM_BYTES;
+            const bool second = lane + 32 < n_chunks;
+            const uint32_t lo = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr)), hi32 = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr) >> 32);
+#pragma unroll 8
+            for (int r = 0; r < LP_HALF; ++r) {
+                const uint64_t pr = (static_cast<uint64_t>(__shfl_sync(0xffffffffu, hi32, r)) << 32) | __shfl_sync(0xffffffffu, lo, r);
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(pr) + lane * 16;
+                const uint32_t bytes = ((valid_mask >> r) & 1u) ? 16u : 0u;
+                const uint32_t swz = static_cast<uint32_t>((r & 7) << 4);
+                cp_async16((dst0 ^ swz) + r * 128, src, bytes);
+                if (second) cp_async16((dst1 ^ swz) + r * 128, src + 512, bytes);
+            }
+            cp_async_commit();
+            row_nxt = resolve(raw_nxt, valid_nxt);                 // page-table load overlaps the copies in flight
+            raw_nxt = load_raw(hi + 2 * LP_GATHER_WARPS);
+            LP_PROF_WAIT(w_group, (cp_async_wait<0>(), true));
+            fence_proxy_async();              // publish the landed rows to the MMA (async) proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->k_full[buf]));
+            row_ptr = row_nxt;
+            valid_cur = valid_nxt;
+        }
+        if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+        if (g == 0 && lane == 0) { LP_PROF_PUT(3, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(4, w_kempty); LP_PROF_PUT(5, w_group); }
+    } else if (warp < LP_SMAX_WARP0) {
+        // ================================================================== exchange: partial logits -> the peer's buffer
+        const int quad = warp & 3;                         // warps 7..10 -> TMEM lane quadrants 3,0,1,2
+        const int h = quad * 32 + lane;
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t peer_xbuf = mapa_shared(smem_u32(xbuf), peer);
+        const uint32_t peer_xfull = mapa_shared(smem_u32(&sh->x_full[0]), peer);
+        bool ok = true;
+        for (int i = 0; i < n_tiles; ++i) {
+            const int b = i & 1;
+            const uint32_t ph = static_cast<uint32_t>(i >> 1) & 1u;
+            // the logits are complete, and the peer has read what this CTA sent two tiles ago into the same buffer
+            ok = mbar_wait(smem_u32(&sh->s_full[b]), ph) && mbar_wait(smem_u32(&sh->x_empty[b]), ph ^ 1u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
+            // [key/4][head][4 keys] fp32: a warp stores 512 contiguous bytes per instruction; every 16 bytes are counted
+            // on the peer's barrier when they land, so nothing here waits for the transfer
+            const uint32_t dst = peer_xbuf + static_cast<uint32_t>(b * LP_XBUF_BYTES + h * 16);
+            const uint32_t bar = peer_xfull + static_cast<uint32_t>(b * 8);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t r[32];
+                tmem_ld32_wait(s_addr + hf * 32, r);
+                if (hf == 1) {   // both halves are in registers: the softmax warps may overwrite the logits with P
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->x_sent[b]));
+                }
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4)
+                    st_async_cluster_f32x4(dst + static_cast<uint32_t>((hf * 8 + j4) * LP_HEADS * 16), __uint_as_float(r[4 * j4]),
+                                           __uint_as_float(r[4 * j4 + 1]), __uint_as_float(r[4 * j4 + 2]), __uint_as_float(r[4 * j4 + 3]), bar);
+            }
+        }
+        if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+    } else {
+        // ================================================================== softmax + output: 4 warps, thread = head
+        const int quad = warp & 3;
+        const int h = quad * 32 + lane;
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        // this CTA's first 256 query dims of this head -> tensor memory, two bf16 per 32-bit column
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DQK + 256 * c);
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                uint32_t r[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint4 u = __ldg(src + a * 8 + v);
+                    r[4 * v + 0] = u.x; r[4 * v + 1] = u.y; r[4 * v + 2] = u.z; r[4 * v + 3] = u.w;
+                }
+                tmem_st32_wait(lane_addr + LP_COL_Q + a * 32, r);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->qt_full));
+        }
+        const float neg_inf = __int_as_float(0xff800000);
+        float m_ref = neg_inf;      // reference maximum (scaled, log2 domain) the exponentials are taken against
+        float l_sum = 0.f;
+        bool ok = true;
+        LP_PROF_DECL(w_sfull); LP_PROF_DECL(w_xfull); LP_PROF_DECL(w_send);
+        LP_PROF_DECL(s_ld); LP_PROF_DECL(s_peer); LP_PROF_DECL(s_arr); LP_PROF_DECL(s_exp); LP_PROF_DECL(s_st);
+        const long long prof_t0 = LP_PROF_NOW();
+        long long seg = prof_t0;
+        (void)seg;
+        const uint32_t peer_xempty = mapa_shared(smem_u32(&sh->x_empty[0]), peer);
+        for (int i = 0; i < n_tiles; ++i) {
+            const int b = i & 1, buf = i % LP_BUFS;
+            const uint32_t ph_k = static_cast<uint32_t>(i / LP_BUFS) & 1u, ph_s = static_cast<uint32_t>(i >> 1) & 1u;
+            // this CTA's exchange barrier for the tile: expect the peer's 32 KB of partial logits
+            if (warp == LP_SMAX_WARP0 && lane == 0) mbar_expect_tx(smem_u32(&sh->x_full[b]), LP_XBUF_BYTES);
+            // k_full is complete long before s_full; waiting on it as well makes the validity masks written by the gather
+            // warps visible to this thread directly rather than through the MMA warp
+            ok = LP_PROF_WAIT(w_sfull, mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
+            float x[LP_TILE];
+            seg = LP_PROF_NOW();
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t r[32];
+                tmem_ld32_wait(s_addr + hf * 32, r);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[hf * 32 + j] = __uint_as_float(r[j]);
+            }
+            LP_PROF_SEG(s_ld, seg);
+            // the peer's partial logits of the same tile (bytes counted as they land: visible once the phase completes)
+            ok = LP_PROF_WAIT(w_xfull, mbar_wait(smem_u32(&sh->x_full[b]), ph_s));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            float tile_max = neg_inf;
+            seg = LP_PROF_NOW();
+            {
+                const float4* xin = reinterpret_cast<const float4*>(xbuf + b * (LP_XBUF_BYTES / 4)) + h;
+#pragma unroll
+                for (int j4 = 0; j4 < LP_TILE / 4; ++j4) {
+                    const float4 pv = xin[j4 * LP_HEADS];
+                    x[4 * j4 + 0] += pv.x; x[4 * j4 + 1] += pv.y; x[4 * j4 + 2] += pv.z; x[4 * j4 + 3] += pv.w;
+                }
+                const uint32_t vm0 = sh->vmask[2 * buf], vm1 = sh->vmask[2 * buf + 1];
+                if ((vm0 & vm1) != 0xffffffffu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        x[j] = ((vm0 >> j) & 1u) ? x[j] : neg_inf;
+                        x[32 + j] = ((vm1 >> j) & 1u) ? x[32 + j] : neg_inf;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < LP_TILE; ++j) tile_max = fmaxf(tile_max, x[j]);
+            }
+            LP_PROF_SEG(s_peer, seg);
+            // the exchange buffer has been read: the peer may send the tile after next into it
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster_relaxed(peer_xempty + static_cast<uint32_t>(b * 8));
+            LP_PROF_SEG(s_arr, seg);
+            tile_max *= p.scale_log2e;                       // softmax_scale > 0
+            // move the reference maximum only when this tile exceeds it by more than 2^8 (or on first use)
+            float corr = 1.f;
+            bool moved = false;
+            if (tile_max > m_ref + 8.f) {
+                moved = (l_sum > 0.f);
+                corr = moved ? lp_exp2(m_ref - tile_max) : 1.f;
+                l_sum *= corr;
+                m_ref = tile_max;
+            }
+            if (__any_sync(0xffffffffu, moved) && i > 0) {
+                // rescale O in tensor memory: the previous tile's P.V must have completed first
+                ok = mbar_wait(smem_u32(&sh->k_empty[(i - 1) % LP_BUFS]), static_cast<uint32_t>((i - 1) / LP_BUFS) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int cc = 0; cc < LP_DVH / 32; ++cc) {
+                    uint32_t o[32];
+                    tmem_ld32_wait(lane_addr + LP_COL_O + cc * 32, o);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * corr);
+                    tmem_st32_wait(lane_addr + LP_COL_O + cc * 32, o);
+                }
+            }
+            const float neg_m = (m_ref == neg_inf) ? 0.f : -m_ref;
+            // P is cut (not rounded) to bf16 with integer ops, which keeps the conversion off the quarter-rate unit the
+            // exponentials already occupy; the row sum adds the very same cut values, so the normalisation stays consistent
+            uint32_t pk[32];
+            float tile_sum = 0.f;
+#pragma unroll
+            for (int j = 0; j < LP_TILE / 2; ++j) {
+                const uint32_t u0 = __float_as_uint(lp_exp2(fmaf(x[2 * j], p.scale_log2e, neg_m))) & 0xffff0000u;
+                const uint32_t u1 = __float_as_uint(lp_exp2(fmaf(x[2 * j + 1], p.scale_log2e, neg_m))) & 0xffff0000u;
+                tile_sum += __uint_as_float(u0) + __uint_as_float(u1);
+                pk[j] = __byte_perm(u0, u1, 0x7632);       // low half = bf16(p0), high half = bf16(p1)
+            }
+            l_sum += tile_sum;
+            LP_PROF_SEG(s_exp, seg);
+            // P overwrites the first 32 columns of the logits: the exchange warps must have read them
+            ok = mbar_wait(smem_u32(&sh->x_sent[b]), ph_s);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tmem_st32_wait(s_addr, pk);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->p_full[b]));
+            LP_PROF_SEG(s_st, seg);
+        }
+        // ---- output: wait for the last P.V, normalise, round to bf16
+        if (ok && n_tiles > 0) {
+            ok = mbar_wait(smem_u32(&sh->k_empty[(n_tiles - 1) % LP_BUFS]), static_cast<uint32_t>((n_tiles - 1) / LP_BUFS) & 1u);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const bool have_o = n_tiles > 0 && __any_sync(0xffffffffu, l_sum > 0.f);   // some P.V has written O
+            uint16_t* orow = p.out + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DV + c * LP_DVH;
+#pragma unroll 1
+            for (int cc = 0; cc < LP_DVH / 32; ++cc) {
+                uint32_t o[32];
+                if (have_o) {
+                    tmem_ld32_wait(lane_addr + LP_COL_O + cc * 32, o);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = 0u;
+                }
+                uint4* dst = reinterpret_cast<uint4*>(orow + cc * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    uint4 u;
+                    u.x = lp_pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                    u.y = lp_pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                    u.z = lp_pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                    u.w = lp_pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                    dst[v] = u;
+                }
+            }
+#ifndef JANUS_ATTN_PROFILE
+            if (p.lse != nullptr && c == 0u)
+                p.lse[static_cast<int64_t>(t) * LP_HEADS + h] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : neg_inf;
+#else
+            if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); }
+#endif
+        } else if (lane == 0) {
+            report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    cluster_sync_all();   // neither CTA leaves while the other may still write into its shared memory or arrive on its barriers
+}
+
+bool sparse_attn_latent_tc_supported(int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
+                                     int64_t tok_stride, int n_kv_heads, int d_v, int k) {
+    if (H_q != LP_HEADS || d_qk != LP_DQK || d_v != LP_DV || n_kv_heads != 1 || k_pool != v_pool) return false;
+    if ((page_stride % 8) != 0 || (tok_stride % 8) != 0 || tok_stride < LP_DQK) return false;
+    if (M > (1 << 30) / LP_HEADS || k <= 0) return false;
+    return true;
+}
+
+int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t page_stride, int64_t tok_stride, const int32_t* idx, int k,
+                                 int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
+                                 float* lse, int32_t* dev_status, cudaStream_t stream) {
+    LpParams p;
+    p.q = static_cast<const uint16_t*>(q);
+    p.pool = static_cast<const uint16_t*>(pool);
+    p.page_stride = page_stride;
+    p.tok_stride = tok_stride;
+    p.idx = idx;
+    p.k = k;
+    p.page_size = page_size;
+    p.page_shift = -1;
+    if ((page_size & (page_size - 1)) == 0) {
+        p.page_shift = 0;
+        while ((1 << p.page_shift) < page_size) ++p.page_shift;
+    }
+    p.page_table = page_table;
+    p.n_logical_pages = n_logical_pages;
+    p.scale_log2e = softmax_scale * 1.4426950408889634f;
+    p.out = static_cast<uint16_t*>(out);
+    p.lse = lse;
+    p.M = M;
+    p.dev_status = dev_status;
+    CUtensorMap tq;
+    if (!make_tmap_2d_sw128(&tq, q, 2, static_cast<uint64_t>(M) * LP_HEADS, LP_DQK, static_cast<uint64_t>(LP_DQK) * 2, LP_HEADS, 64))
+        return JANUS_ERR_CUDA;
+    const size_t smem = LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES + LP_Q_ATOM_BYTES + sizeof(LpShared) + 16;
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(sparse_attn_latent_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    sparse_attn_latent_pair_kernel<<<2 * M, LP_THREADS, smem, stream>>>(tq, p);   // clusters of 2 CTAs (compile-time cluster dims)
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
+
+}  // namespace janus
