@@ -16,7 +16,7 @@
 namespace janus {
 
 constexpr int TK_THREADS = 512;
-constexpr int TK_CAP = 12288;       // candidate slots (key + index = 8 bytes each)
+constexpr int TK_CAP = 8192;        // candidate slots (key + index = 8 bytes each); 73 KB per CTA keeps three CTAs on an SM
 constexpr int TK_BUCKETS = 2048;
 constexpr int TK_SAMPLE = 4096;     // 512 threads x 8 floats (one 32-byte sector each)
 
