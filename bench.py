@@ -82,6 +82,17 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def captured_traffic(kernel_key: str, rows: int):
+    """DRAM bytes of one launch of `kernel_key`, from the ncu capture summarised under profiles/ (a small case of the same
+    kernel), scaled by query rows to this launch.  None if no capture is recorded."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    d = json.load(open(p))
+    b = d.get("dram_bytes_per_launch", {}).get(kernel_key)
+    return None if b is None else b * rows / d["rows_in_capture"]
+
+
 def workload_numbers(shp):
     """Algorithmic work of one step (exact pass), per the definitions in the design doc."""
     L, M, S = shp.L, shp.M, shp.S
@@ -339,16 +350,19 @@ def main():
     dom = int(np.argmax(mean_ms))
     if names[dom] == "indexer_scores":
         roofline = {"kernel": "indexer_tc_kernel", "bound": "tensor", "achieved": kernels["indexer_scores"]["tflops"], "peak": tensor_peak_idx,
-                    "unit": "TFLOP/s", "frac": kernels["indexer_scores"]["frac_tensor_peak"], "traffic": None,
+                    "unit": "TFLOP/s", "frac": kernels["indexer_scores"]["frac_tensor_peak"],
+                    "traffic": captured_traffic("indexer_tc" if fp8 else "indexer_tc_bf16", shp.M),
+                    "traffic_note": "ncu dram bytes of a 296-row capture of the same kernel scaled by rows (profiles/); for bf16 the capture is at L=32768",
                     "peak_source": f"{peaks['source']} bf16 sustained" + (" x2 (nominal fp8:bf16 ratio)" if fp8 else "")}
     elif names[dom] == "sparse_attn_prefill":
         roofline = {"kernel": "sparse_attn", "bound": "tensor", "achieved": kernels["sparse_attn_prefill"]["tflops"],
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": kernels["sparse_attn_prefill"]["frac_tensor_peak"],
-                    "traffic": None, "peak_source": f"{peaks['source']} bf16 sustained"}
+                    "traffic": captured_traffic("sparse_attn_latent", shp.M), "peak_source": f"{peaks['source']} bf16 sustained"}
     else:
         key = names[dom]
         roofline = {"kernel": key, "bound": "hbm", "achieved": kernels[key]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": kernels[key]["gbs"] / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth"}
+                    "frac": kernels[key]["gbs"] / peaks["hbm_gbs"], "traffic": captured_traffic("topk_rows" if key == "topk" else "page_mark", shp.M),
+                    "peak_source": f"{peaks['source']} copy bandwidth"}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
