@@ -137,6 +137,15 @@ int janus_page_demand(const int32_t* idx, int64_t n_rows, int k,
                       void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * Union of page sets - synchronisation-free parallel prediction (Sec. 4.2, Eq. 3): the history is cut into disjoint
+ * shards, every shard selects its own top-(k/N) and builds its own page set with janus_page_demand; the predicted set
+ * the exact pass is compared against is the union of the per-shard sets.
+ *
+ *     dst |= src        (both bitmaps of n_phys_pages bits, as written by janus_page_demand)
+ */
+int janus_page_union(uint32_t* dst, const uint32_t* src, int64_t n_phys_pages, void* stream);
+
+/*
  * Sparse attention over the selected rows only (Sec. 2.2, "core attention"):
  *
  *     out[t, h, :] = sum_{s in idx[t]} softmax_s( softmax_scale * < q[t, h, :d_qk], K_s[:d_qk] > ) * V_s[:d_v]

@@ -25,7 +25,7 @@ EXPORTS = [
     "janus_version", "janus_last_cuda_error",
     "janus_indexer_scores_workspace_size", "janus_indexer_scores",
     "janus_topk_workspace_size", "janus_topk",
-    "janus_page_demand_workspace_size", "janus_page_demand",
+    "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
 ]
 
@@ -62,6 +62,8 @@ def load() -> ctypes.CDLL:
     lib.janus_page_demand.restype = c_i
     lib.janus_page_demand.argtypes = [c_p, c_i64, c_i, c_i64, c_i, c_p, c_i64, c_i64, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p,
                                       c_i64, c_p, c_sz, c_p, c_p]
+    lib.janus_page_union.restype = c_i
+    lib.janus_page_union.argtypes = [c_p, c_p, c_i64, c_p]
     lib.janus_sparse_attn_prefill_workspace_size.restype = c_sz
     lib.janus_sparse_attn_prefill_workspace_size.argtypes = [c_i, c_i, c_i, c_i, c_i]
     lib.janus_sparse_attn_prefill.restype = c_i
@@ -187,6 +189,12 @@ def janus_page_demand(idx: torch.Tensor, *, demand_limit: int, page_size: int, p
                                _ptr(out["runs"]), cp + 4, *miss_args, cap, None, 0, _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_page_demand")
     return out
+
+
+def janus_page_union(dst: torch.Tensor, src: torch.Tensor, n_phys_pages: int) -> torch.Tensor:
+    """dst |= src for two page bitmaps written by janus_page_demand (union of per-shard predicted sets, Sec. 4.2)."""
+    _check(load().janus_page_union(_ptr(dst), _ptr(src), int(n_phys_pages), _stream()), "janus_page_union")
+    return dst
 
 
 def janus_sparse_attn_prefill(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, idx: torch.Tensor, *,

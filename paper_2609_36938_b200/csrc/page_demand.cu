@@ -135,7 +135,22 @@ page_lists_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restric
                         dev_status, scan_scratch);
 }
 
+__global__ void page_union_kernel(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, int n_words) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += gridDim.x * blockDim.x) dst[i] |= src[i];
+}
+
 }  // namespace janus
+
+extern "C" int janus_page_union(uint32_t* dst, const uint32_t* src, int64_t n_phys_pages, void* stream_) {
+    using namespace janus;
+    if (!dst || !src || n_phys_pages <= 0) return JANUS_ERR_INVALID_ARG;
+    if (n_phys_pages > (int64_t(1) << 31) - 64) return JANUS_ERR_UNSUPPORTED;
+    const int n_words = static_cast<int>((n_phys_pages + 31) / 32);
+    const int blocks = n_words < 256 * 148 ? (n_words + 255) / 256 : 148;
+    page_union_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream_)>>>(dst, src, n_words);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
 
 extern "C" size_t janus_page_demand_workspace_size(int64_t, int, int64_t) { return 0; }
 
