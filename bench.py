@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-fused", action="store_true", help="skip the side measurement of janus_indexer_topk")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     args.steps_ref = max(1, min(args.steps, 3))
@@ -324,6 +325,33 @@ def main():
         e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
                "ms_per_step": e2e_ms, "inputs": "all operands (queries, keys, weights, Q, KV pool, page table) uploaded every step"}
 
+    # ---- side measurement (not part of `value`): indexer + top-k as one call that never stores the score matrix
+    fused = None
+    if not args.no_fused:
+        lib = B.load()
+        ws_bytes = int(lib.janus_indexer_topk_workspace_size(shp.M, shp.H_I, shp.D_I, shp.S, shp.L, 1, 1 if shp.idx_dtype == "fp8" else 0, shp.k))
+        del scores
+        torch.cuda.empty_cache()
+        ws = torch.empty((ws_bytes,), dtype=torch.uint8, device="cuda")
+        fidx = torch.empty((shp.M, shp.k), dtype=torch.int32, device="cuda")
+
+        def fused_call():
+            B.janus_indexer_topk(d["q_idx"], d["k_idx"], d["w"], shp.k, q_scale=d["q_scale"], k_scale=d["k_scale"], row_bias=d["row_bias"],
+                                 col_bias=d["col_bias"], q_pos0=shp.L, causal=True, workspace=ws, idx=fidx, want_count=False, want_kth=False)
+
+        for _ in range(3):
+            fused_call()
+        barrier()
+        f0, f1 = ev(), ev()
+        f0.record(stream)
+        for _ in range(5):
+            fused_call()
+        f1.record(stream)
+        barrier()
+        B.check_dev_status()
+        fused = {"ms": f0.elapsed_time(f1) / 5, "two_call_ms": float(per_call[:, 0].mean() + per_call[:, 1].mean()), "workspace_bytes": ws_bytes,
+                 "score_matrix_bytes": int(shp.M) * int(ld) * 4}
+
     clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
@@ -375,6 +403,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3+bf16" if fp8 else "bf16", "data": "synthetic",
         "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
         "kernels": {k: {kk: (round(float(vv), 4)) for kk, vv in v.items()} for k, v in kernels.items()},
+        "indexer_topk_one_call": fused,
         "page_demand": {"n_pages": int(counts[0]), "n_runs": int(counts[1]), "n_miss": int(counts[2]), "n_miss_runs": int(counts[3])},
     }
     print(json.dumps(line))

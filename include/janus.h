@@ -105,6 +105,30 @@ int janus_topk(const float* scores, int64_t scores_ld, int M, int64_t n_keys,
                void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * Indexer scores and per-row top-k in one call - Eq. 1 (Sec. 2.2) without the [M, n_keys] score matrix in memory.
+ * Same operands and semantics as janus_indexer_scores followed by janus_topk (same masking, same tie freedom, same
+ * outputs idx / count / kth); scores only ever exist as short per-row candidate lists in the workspace.
+ * A sampled estimate of each row's k-th score decides which scores the indexer keeps; rows the estimate misjudges are
+ * recomputed exactly, so the result never depends on the sample.  Shapes the tensor-core indexer does not take (and
+ * head counts other than 64, or 32 with 256-byte rows), fewer than 16384 keys visible to every row, k > 4096 or more
+ * than 8192 keys beyond the first row's prefix run the two calls internally with the scores in the workspace.
+ *
+ *   ws   device scratch of at least janus_indexer_topk_workspace_size(...) bytes, 16-byte aligned; contents undefined on
+ *        return; two calls sharing a workspace must not overlap on the device.
+ */
+size_t janus_indexer_topk_workspace_size(int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal, int dtype, int k);
+int janus_indexer_topk(const void* q_idx, int64_t q_stride_tok,
+                       const void* k_idx, int64_t k_stride_tok,
+                       const float* w,
+                       const float* q_scale, int64_t q_scale_stride_tok,
+                       const float* k_scale,
+                       const float* row_bias, const float* col_bias,
+                       int M, int H_I, int D_I, int64_t n_keys,
+                       int64_t q_pos0, int causal, int dtype, int k,
+                       int32_t* idx, int32_t* count, float* kth,
+                       void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/*
  * Page demand - union of the selections (Sec. 2.2), best-effort read packing into maximal runs of physically
  * adjacent pages (Sec. 4.3) and the corrective-read set "exact minus predicted" (Sec. 4.2).
  *

@@ -25,6 +25,7 @@ EXPORTS = [
     "janus_version", "janus_last_cuda_error",
     "janus_indexer_scores_workspace_size", "janus_indexer_scores",
     "janus_topk_workspace_size", "janus_topk",
+    "janus_indexer_topk_workspace_size", "janus_indexer_topk",
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
 ]
@@ -57,6 +58,11 @@ def load() -> ctypes.CDLL:
     lib.janus_topk_workspace_size.argtypes = [c_i, c_i64, c_i]
     lib.janus_topk.restype = c_i
     lib.janus_topk.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p, c_p]
+    lib.janus_indexer_topk_workspace_size.restype = c_sz
+    lib.janus_indexer_topk_workspace_size.argtypes = [c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i]
+    lib.janus_indexer_topk.restype = c_i
+    lib.janus_indexer_topk.argtypes = [c_p, c_i64, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i,
+                                       c_p, c_p, c_p, c_p, c_sz, c_p, c_p]
     lib.janus_page_demand_workspace_size.restype = c_sz
     lib.janus_page_demand_workspace_size.argtypes = [c_i64, c_i, c_i64]
     lib.janus_page_demand.restype = c_i
@@ -160,6 +166,35 @@ def janus_topk(scores: torch.Tensor, n_keys: int, k: int, *, q_pos0: int = 0, ca
     rc = lib.janus_topk(_ptr(scores), scores.stride(0), M, int(n_keys), int(q_pos0), int(bool(causal)), int(k), _ptr(idx), _ptr(count),
                         _ptr(kth), None, 0, _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_topk")
+    return idx, count, kth
+
+
+def janus_indexer_topk(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, k: int, *, q_scale: Optional[torch.Tensor] = None,
+                       k_scale: Optional[torch.Tensor] = None, row_bias: Optional[torch.Tensor] = None,
+                       col_bias: Optional[torch.Tensor] = None, q_pos0: int = 0, causal: bool = True, want_count: bool = True,
+                       want_kth: bool = True, workspace: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None):
+    """Indexer scores and per-row top-k in one call, without the score matrix.  Returns (idx [M,k], count | None, kth | None).
+    `workspace` (uint8 CUDA tensor) is allocated if not given or too small; pass one to reuse it across calls; `idx` likewise."""
+    lib = load()
+    M, H, D = q_idx.shape
+    n_keys = k_idx.shape[0]
+    dtype = _idx_dtype_code(q_idx)
+    if _idx_dtype_code(k_idx) != dtype:
+        raise JanusError("q_idx and k_idx must share a dtype")
+    need = int(lib.janus_indexer_topk_workspace_size(M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype, int(k)))
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty((max(need, 16),), dtype=torch.uint8, device=q_idx.device)
+    if idx is None:
+        idx = torch.empty((M, k), dtype=torch.int32, device=q_idx.device)
+    elif idx.shape != (M, k) or idx.dtype != torch.int32 or not idx.is_contiguous():
+        raise JanusError("idx must be a contiguous [M, k] int32 tensor")
+    count = torch.empty((M,), dtype=torch.int32, device=q_idx.device) if want_count else None
+    kth = torch.empty((M,), dtype=torch.float32, device=q_idx.device) if want_kth else None
+    qs_stride = H if (q_scale is not None and q_scale.dim() == 2) else 0
+    rc = lib.janus_indexer_topk(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
+                                _ptr(row_bias), _ptr(col_bias), M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype, int(k), _ptr(idx),
+                                _ptr(count), _ptr(kth), _ptr(workspace), workspace.numel(), _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_indexer_topk")
     return idx, count, kth
 
 

@@ -46,6 +46,21 @@ struct TcParams {
     int32_t* dev_status;
 };
 
+// Candidate mode (fused indexer + top-k): instead of storing scores, every visible score >= thr[t] is appended to row t's
+// candidate list; `scores` is unused.  A kernel parameter of its own: the score-matrix kernel's code does not depend on it.
+struct TcCandParams {
+    const float* thr;     // [M] per-row thresholds
+    int32_t* cand_cnt;    // [M] candidates appended so far (may exceed cand_cap: only the first cand_cap are stored)
+    int2* cand;           // [M, cand_cap] (score bits, key index)
+    int cand_cap;
+};
+
+// Candidate mode stages appends in shared memory: each epilogue warp owns, for each of its (at most TC_CAND_TPW) tokens,
+// TC_CAND_SLOTS (score, key) slots, and moves a full set to the row's global list with one counter update.
+constexpr int TC_CAND_TPW = 8;
+constexpr int TC_CAND_SLOTS = 32;
+constexpr int TC_CAND_STAGE_BYTES = 8 * TC_CAND_TPW * TC_CAND_SLOTS * static_cast<int>(sizeof(int2));
+
 struct TcBarriers {
     uint64_t q_full;
     uint64_t k_full[TC_MAX_STAGES];
@@ -86,9 +101,9 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
     }
 }
 
-template <int H, bool FP8>
+template <int H, bool FP8, bool CAND>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p) {
+indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p, const TcCandParams cp) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int TPS = TC_N / H;                      // tokens per query sub-tile
     const int atoms = p.atoms, nq = p.nq, stages = p.stages;
@@ -98,7 +113,9 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     unsigned char* k_smem = smem + nq * q_sub_bytes;
     float* ws = reinterpret_cast<float*>(k_smem + stages * k_stage_bytes);   // [nq*256] w * q_scale, column order
     float* rbs = ws + nq * TC_N;                                             // [nq*TPS] row_bias of this CTA's tokens
-    TcBarriers* bars = reinterpret_cast<TcBarriers*>(rbs + nq * TPS);
+    float* thrs = rbs + nq * TPS;                                            // [nq*TPS] candidate thresholds of this CTA's tokens
+    int2* cstage = reinterpret_cast<int2*>(thrs + nq * TPS);                 // candidate staging (candidate mode only)
+    TcBarriers* bars = reinterpret_cast<TcBarriers*>(reinterpret_cast<unsigned char*>(cstage) + (CAND ? TC_CAND_STAGE_BYTES : 0));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tpc = nq * TPS;                                   // tokens per CTA
@@ -145,7 +162,10 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
         ws[n] = v;
     }
-    for (int n = threadIdx.x; n < tpc; n += TC_THREADS) rbs[n] = (p.row_bias != nullptr && t0 + n < p.M) ? p.row_bias[t0 + n] : 0.f;
+    for (int n = threadIdx.x; n < tpc; n += TC_THREADS) {
+        rbs[n] = (p.row_bias != nullptr && t0 + n < p.M) ? p.row_bias[t0 + n] : 0.f;
+        if constexpr (CAND) thrs[n] = t0 + n < p.M ? cp.thr[t0 + n] : 0.f;
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -219,6 +239,17 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         const int quad = warp & 3;              // TMEM lanes 32*quad .. 32*quad+31
         const float neg_inf = __int_as_float(0xff800000);
         bool ok = true;
+        // candidate staging of this warp: lane i keeps the fill count of the warp's token slot i
+        int2* my_stage = cstage + (warp - 2) * TC_CAND_TPW * TC_CAND_SLOTS;
+        int cand_fill = 0;
+        auto cand_flush = [&](int slot, int t, int c) {
+            __syncwarp();                                        // the staged entries were written by other lanes
+            int base = 0;
+            if (lane == 0) base = atomicAdd(cp.cand_cnt + t, c);
+            base = __shfl_sync(0xffffffffu, base, 0);
+            if (lane < c && base + lane < cp.cand_cap) cp.cand[static_cast<int64_t>(t) * cp.cand_cap + base + lane] = my_stage[slot * TC_CAND_SLOTS + lane];
+            __syncwarp();                                        // slots are free again
+        };
         for (int it = 0; it < n_vis && ok; ++it) {
             const int64_t s = static_cast<int64_t>(tile_begin + it) * TC_KEYS + quad * 32 + lane;
             const bool key_ok = s < p.n_keys;
@@ -234,11 +265,28 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 auto store = [&](int tt, float v) {
                     const int t = tsub0 + tt;
-                    if (t < p.M && key_ok) {
+                    if constexpr (!CAND) {
+                        if (t < p.M && key_ok) {
+                            float out = v * kscale;
+                            out = fmaf(rbs[j * TPS + tt], cb, out);
+                            if (p.causal && s > p.q_pos0 + t) out = neg_inf;
+                            p.scores[static_cast<int64_t>(t) * p.ld + s] = out;
+                        }
+                    } else {
+                        // all 32 lanes (32 consecutive keys of one token) get here together
                         float out = v * kscale;
                         out = fmaf(rbs[j * TPS + tt], cb, out);
-                        if (p.causal && s > p.q_pos0 + t) out = neg_inf;
-                        p.scores[static_cast<int64_t>(t) * p.ld + s] = out;
+                        const bool masked = p.causal && s > p.q_pos0 + t;
+                        const bool pass = t < p.M && key_ok && !masked && out >= thrs[j * TPS + tt];
+                        const uint32_t m = __ballot_sync(0xffffffffu, pass);
+                        if (m != 0u) {
+                            const int slot = (j >> 1) * TPS + tt;
+                            int c = __shfl_sync(0xffffffffu, cand_fill, slot);
+                            const int n = __popc(m);
+                            if (c + n > TC_CAND_SLOTS) { cand_flush(slot, t, c); c = 0; }
+                            if (pass) my_stage[slot * TC_CAND_SLOTS + c + __popc(m & ((1u << lane) - 1u))] = make_int2(__float_as_int(out), static_cast<int>(s));
+                            if (lane == slot) cand_fill = c + n;
+                        }
                     }
                 };
                 // two register buffers: the load of the next 32 columns is in flight while this one is reduced
@@ -263,8 +311,14 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             }
         }
         if (!ok && lane == 0) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }
-        // key tiles no token of this CTA may see: -inf
-        for (int tile = vis_end + e; tile < tile_end; tile += 2) {
+        if (CAND) {
+            for (int slot = 0; slot < TC_CAND_TPW; ++slot) {
+                const int c = __shfl_sync(0xffffffffu, cand_fill, slot);
+                if (c > 0) cand_flush(slot, t0 + (2 * (slot / TPS) + e) * TPS + slot % TPS, c);
+            }
+        }
+        // key tiles no token of this CTA may see: -inf (score-matrix mode only)
+        for (int tile = vis_end + e; !CAND && tile < tile_end; tile += 2) {
             const int64_t s = static_cast<int64_t>(tile) * TC_KEYS + quad * 32 + lane;
             if (s < p.n_keys)
                 for (int t = t0; t <= t_hi; ++t) p.scores[static_cast<int64_t>(t) * p.ld + s] = neg_inf;
@@ -312,10 +366,18 @@ bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_
     return true;
 }
 
-template <int H, bool FP8>
-static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
-    JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    indexer_tc_kernel<H, FP8><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p);
+// Candidate mode needs every epilogue warp's tokens to fit its staging slots, whatever sub-tile count the launch picks.
+bool indexer_tc_candidates_supported(int H, int D, int dtype) {
+    const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
+    const int nq_max = row_bytes == 128 ? 4 : 2;
+    return (H == 32 || H == 64) && (nq_max / 2) * (TC_N / H) <= TC_CAND_TPW;
+}
+
+template <int H, bool FP8, bool CAND>
+static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, const TcCandParams& cp, dim3 grid, size_t smem,
+                     cudaStream_t stream) {
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8, CAND>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    indexer_tc_kernel<H, FP8, CAND><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p, cp);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
@@ -323,20 +385,24 @@ static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParam
 int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok, const float* w, const float* q_scale,
                       int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int M, int H,
                       int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype, float* scores, int64_t ld, int32_t* dev_status,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, const float* thr, int32_t* cand_cnt, void* cand, int cand_cap) {
     const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3;
     const int esz = fp8 ? 1 : 2;
     TcParams p;
     p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
     p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = ld; p.n_keys = n_keys; p.q_pos0 = q_pos0;
     p.M = M; p.H = H; p.causal = causal; p.dev_status = dev_status;
+    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap};
     p.atoms = D * esz / 128;
     p.nq = p.atoms == 1 ? 4 : 2;
     const int tps = TC_N / H;
     while (p.nq > 2 && static_cast<int64_t>(p.nq / 2) * tps >= M) p.nq /= 2;   // small M: do not load empty sub-tiles
     const int q_bytes = p.nq * p.atoms * TC_N * 128;
     const int k_stage = p.atoms * TC_KEYS * 128;
-    const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + p.nq * tps) + static_cast<int>(sizeof(TcBarriers)) + 16;
+    const bool cand_mode = thr != nullptr;
+    if (cand_mode && (p.nq + 1) / 2 * tps > TC_CAND_TPW) return JANUS_ERR_UNSUPPORTED;
+    const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + 2 * p.nq * tps) + (cand_mode ? TC_CAND_STAGE_BYTES : 0) +
+                     static_cast<int>(sizeof(TcBarriers)) + 16;
     p.stages = (TC_SMEM_BUDGET - q_bytes - tail) / k_stage;
     if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
     if (p.stages < 2) return JANUS_ERR_UNSUPPORTED;
@@ -357,15 +423,22 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(n_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols))
         return JANUS_ERR_CUDA;
 
-#define JANUS_TC_CASE(HH)                                                             \
+#define JANUS_TC_CASE(HH, CC)                                                         \
     case HH:                                                                          \
-        return fp8 ? launch_tc<HH, true>(tq, tk, p, grid, smem, stream) : launch_tc<HH, false>(tq, tk, p, grid, smem, stream);
+        return fp8 ? launch_tc<HH, true, CC>(tq, tk, p, cp, grid, smem, stream) : launch_tc<HH, false, CC>(tq, tk, p, cp, grid, smem, stream);
+    if (cand_mode) {
+        switch (H) {   // head counts whose tokens per epilogue warp fit the staging slots
+            JANUS_TC_CASE(32, true)
+            JANUS_TC_CASE(64, true)
+        }
+        return JANUS_ERR_UNSUPPORTED;
+    }
     switch (H) {
-        JANUS_TC_CASE(4)
-        JANUS_TC_CASE(8)
-        JANUS_TC_CASE(16)
-        JANUS_TC_CASE(32)
-        JANUS_TC_CASE(64)
+        JANUS_TC_CASE(4, false)
+        JANUS_TC_CASE(8, false)
+        JANUS_TC_CASE(16, false)
+        JANUS_TC_CASE(32, false)
+        JANUS_TC_CASE(64, false)
     }
 #undef JANUS_TC_CASE
     return JANUS_ERR_UNSUPPORTED;

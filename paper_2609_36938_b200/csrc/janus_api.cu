@@ -17,7 +17,7 @@ bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_
 int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok, const float* w, const float* q_scale,
                       int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int M, int H,
                       int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype, float* scores, int64_t ld, int32_t* dev_status,
-                      cudaStream_t stream);
+                      cudaStream_t stream, const float* thr = nullptr, int32_t* cand_cnt = nullptr, void* cand = nullptr, int cand_cap = 0);
 
 int launch_sparse_attn_generic(const void* q, int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
                                int64_t tok_stride, int64_t head_stride, int n_kv_heads, int d_v, const int32_t* idx, int k,
@@ -29,6 +29,29 @@ bool sparse_attn_latent_tc_supported(int M, int H_q, int d_qk, const void* k_poo
 int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t page_stride, int64_t tok_stride, const int32_t* idx, int k,
                                  int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
                                  float* lse, int32_t* dev_status, cudaStream_t stream);
+
+// Host-side checks shared by the entry points that take indexer operands.  JANUS_OK also for empty problems.
+int validate_indexer_args(const void* q_idx, int64_t q_stride_tok, const void* k_idx, int64_t k_stride_tok, const float* w,
+                          const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
+                          const float* col_bias, int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int dtype) {
+    if (M < 0 || H_I <= 0 || D_I <= 0 || n_keys < 0 || q_pos0 < 0) return JANUS_ERR_INVALID_ARG;
+    if (dtype != JANUS_DTYPE_BF16 && dtype != JANUS_DTYPE_FP8_E4M3) return JANUS_ERR_UNSUPPORTED;
+    if ((D_I % 16) != 0) return JANUS_ERR_UNSUPPORTED;
+    if (M == 0 || n_keys == 0) return JANUS_OK;
+    const int esz = dtype == JANUS_DTYPE_BF16 ? 2 : 1;
+    if (!q_idx || !k_idx || !w) return JANUS_ERR_INVALID_ARG;
+    if (!aligned16(q_idx) || !aligned16(k_idx)) return JANUS_ERR_INVALID_ARG;
+    if (q_stride_tok < static_cast<int64_t>(H_I) * D_I || k_stride_tok < D_I) return JANUS_ERR_INVALID_ARG;
+    if ((q_stride_tok * esz) % 16 != 0 || (k_stride_tok * esz) % 16 != 0) return JANUS_ERR_INVALID_ARG;
+    if ((row_bias == nullptr) != (col_bias == nullptr)) return JANUS_ERR_INVALID_ARG;
+    if (dtype == JANUS_DTYPE_FP8_E4M3) {
+        if (!q_scale || !k_scale) return JANUS_ERR_INVALID_ARG;
+        if (q_scale_stride_tok != 0 && q_scale_stride_tok != H_I) return JANUS_ERR_INVALID_ARG;
+    } else if (q_scale || k_scale) {
+        return JANUS_ERR_INVALID_ARG;
+    }
+    return JANUS_OK;
+}
 
 }  // namespace janus
 
@@ -45,23 +68,12 @@ extern "C" int janus_indexer_scores(const void* q_idx, int64_t q_stride_tok, con
                                     int32_t* dev_status, void* stream_) {
     using namespace janus;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (M < 0 || H_I <= 0 || D_I <= 0 || n_keys < 0 || q_pos0 < 0) return JANUS_ERR_INVALID_ARG;
-    if (dtype != JANUS_DTYPE_BF16 && dtype != JANUS_DTYPE_FP8_E4M3) return JANUS_ERR_UNSUPPORTED;
-    if ((D_I % 16) != 0) return JANUS_ERR_UNSUPPORTED;
+    const int vrc = validate_indexer_args(q_idx, q_stride_tok, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias,
+                                          M, H_I, D_I, n_keys, q_pos0, dtype);
+    if (vrc != JANUS_OK) return vrc;
     if (M == 0 || n_keys == 0) return JANUS_OK;
-    const int esz = dtype == JANUS_DTYPE_BF16 ? 2 : 1;
-    if (!q_idx || !k_idx || !w || !scores) return JANUS_ERR_INVALID_ARG;
-    if (!aligned16(q_idx) || !aligned16(k_idx) || !aligned16(scores)) return JANUS_ERR_INVALID_ARG;
-    if (q_stride_tok < static_cast<int64_t>(H_I) * D_I || k_stride_tok < D_I) return JANUS_ERR_INVALID_ARG;
-    if ((q_stride_tok * esz) % 16 != 0 || (k_stride_tok * esz) % 16 != 0) return JANUS_ERR_INVALID_ARG;
+    if (!scores || !aligned16(scores)) return JANUS_ERR_INVALID_ARG;
     if (scores_ld < n_keys || (scores_ld & 3) != 0) return JANUS_ERR_INVALID_ARG;
-    if ((row_bias == nullptr) != (col_bias == nullptr)) return JANUS_ERR_INVALID_ARG;
-    if (dtype == JANUS_DTYPE_FP8_E4M3) {
-        if (!q_scale || !k_scale) return JANUS_ERR_INVALID_ARG;
-        if (q_scale_stride_tok != 0 && q_scale_stride_tok != H_I) return JANUS_ERR_INVALID_ARG;
-    } else if (q_scale || k_scale) {
-        return JANUS_ERR_INVALID_ARG;
-    }
     // debugging aid: JANUS_FORCE_GENERAL_INDEXER=1 routes every shape to the general kernel
     const char* force_general = getenv("JANUS_FORCE_GENERAL_INDEXER");
     if (!(force_general && force_general[0] == '1') && indexer_tc_supported(M, H_I, D_I, n_keys, q_stride_tok, k_stride_tok, dtype))

@@ -11,235 +11,22 @@
 // If the sample misjudges the row (fewer than k candidates, or more than the buffer holds) the
 // same exact selection runs over the row in global memory instead; that path is slower, never
 // wrong.  Rows that fit the buffer skip the sampling step.
-#include "janus_common.cuh"
+#include "topk_select.cuh"
 
 namespace janus {
 
-constexpr int TK_THREADS = 512;
-constexpr int TK_CAP = 8192;        // candidate slots (key + index = 8 bytes each); 73 KB per CTA keeps three CTAs on an SM
-constexpr int TK_BUCKETS = 2048;
-constexpr int TK_SAMPLE = 4096;     // 512 threads x 8 floats (one 32-byte sector each)
-
-struct TopkShared {
-    uint32_t cand_key[TK_CAP];
-    int32_t cand_idx[TK_CAP];
-    int hist[TK_BUCKETS];
-    int scan[40];
-    int n_cand;
-    int out_pos;
-    int eq_taken;
-    uint32_t red_lo, red_hi;
-    int sel_bucket, sel_above;
-};
-
-struct SmemSource {
-    const uint32_t* key;
-    const int32_t* idx;
-    int n;
-    __device__ __forceinline__ int size() const { return n; }
-    __device__ __forceinline__ uint32_t key_at(int i) const { return key[i]; }
-    __device__ __forceinline__ int32_t idx_at(int i) const { return idx ? idx[i] : i; }
-};
-struct GlobalSource {
-    const float* row;
-    int n;
-    __device__ __forceinline__ int size() const { return n; }
-    __device__ __forceinline__ uint32_t key_at(int i) const { return float_to_key(__ldcg(row + i)); }
-    __device__ __forceinline__ int32_t idx_at(int i) const { return i; }
-};
-
-// Exact `need`-th largest key of a source (1 <= need <= number of elements).
-// Returns the threshold key T and, in *n_eq_take, how many elements equal to T belong to the selection.
-// Every thread of the CTA must call it; results are uniform.
-template <class Src>
-__device__ uint32_t select_kth(const Src& src, int need, TopkShared& sh, int* n_eq_take) {
-    const int tid = threadIdx.x;
-    const int n = src.size();
-    // range of the active keys
-    uint32_t lo = 0xffffffffu, hi = 0u;
-    for (int i = tid; i < n; i += TK_THREADS) {
-        const uint32_t key = src.key_at(i);
-        lo = min(lo, key);
-        hi = max(hi, key);
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, d));
-        hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, d));
-    }
-    if (tid == 0) { sh.red_lo = 0xffffffffu; sh.red_hi = 0u; }
-    __syncthreads();
-    if ((tid & 31) == 0) { atomicMin(&sh.red_lo, lo); atomicMax(&sh.red_hi, hi); }
-    __syncthreads();
-    lo = sh.red_lo;
-    hi = sh.red_hi;
-    __syncthreads();
-
-    for (int iter = 0; iter < 8 && lo < hi; ++iter) {
-        const uint32_t range = hi - lo;
-        const int bits = 32 - __clz(range);                   // range < 2^bits
-        const int shift = bits > 11 ? bits - 11 : 0;          // (range >> shift) < 2048
-        for (int i = tid; i < TK_BUCKETS; i += TK_THREADS) sh.hist[i] = 0;
-        __syncthreads();
-        for (int i = tid; i < n; i += TK_THREADS) {
-            const uint32_t key = src.key_at(i);
-            if (key >= lo && key <= hi) atomicAdd(&sh.hist[(key - lo) >> shift], 1);
-        }
-        __syncthreads();
-        // walk the buckets from the top: thread t owns the 4 buckets 2047-4t .. 2044-4t
-        int c[4];
-        int mine = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { c[j] = sh.hist[TK_BUCKETS - 1 - (4 * tid + j)]; mine += c[j]; }
-        int total;
-        int above = block_exclusive_scan<TK_THREADS>(mine, sh.scan, &total);
-        if (above < need && need <= above + mine) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (above < need && need <= above + c[j]) { sh.sel_bucket = TK_BUCKETS - 1 - (4 * tid + j); sh.sel_above = above; }
-                above += c[j];
-            }
-        }
-        __syncthreads();
-        const uint32_t b = static_cast<uint32_t>(sh.sel_bucket);
-        need -= sh.sel_above;
-        const uint32_t new_lo = lo + (b << shift);
-        if (b < (range >> shift)) hi = new_lo + ((1u << shift) - 1u);   // the top bucket keeps hi (and cannot overflow)
-        lo = new_lo;
-        __syncthreads();
-    }
-    *n_eq_take = need;   // lo == hi: `need` of the elements equal to lo complete the selection
-    return lo;
-}
-
-// Writes the selection (all keys > T, plus n_eq of the keys == T) to out[0..k).
-template <class Src>
-__device__ void emit_selection(const Src& src, uint32_t T, int n_eq, int32_t* out, TopkShared& sh) {
-    const int n = src.size();
-    for (int i = threadIdx.x; i < n; i += TK_THREADS) {
-        const uint32_t key = src.key_at(i);
-        if (key > T) {
-            out[atomicAdd(&sh.out_pos, 1)] = src.idx_at(i);
-        } else if (key == T) {
-            if (atomicAdd(&sh.eq_taken, 1) < n_eq) out[atomicAdd(&sh.out_pos, 1)] = src.idx_at(i);
-        }
-    }
-}
-
-// Keeps x (at row position i) if it is at or above the streaming threshold.  The float comparison admits a superset of
-// the exact key comparison (it treats -0 and +0 alike); the exact selection afterwards works on keys.
-__device__ __forceinline__ void keep_if_candidate(float x, int i, float thr_f, TopkShared& sh) {
-    if (x >= thr_f) {
-        const int pos = atomicAdd(&sh.n_cand, 1);
-        if (pos < TK_CAP) { sh.cand_key[pos] = float_to_key(x); sh.cand_idx[pos] = i; }
-    }
-}
+constexpr int TK_CAP = 8192;        // 73 KB of shared memory per CTA keeps three CTAs on an SM
+using TopkShared = TopkSharedT<TK_CAP>;
 
 __global__ void __launch_bounds__(TK_THREADS)
 topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int k,
                  int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-    const int tid = threadIdx.x;
     const int t = blockIdx.x;
-    const float* row = scores + static_cast<int64_t>(t) * ld;
-    int32_t* out = idx + static_cast<int64_t>(t) * k;
     int64_t prefix64 = causal ? min(n_keys, q_pos0 + t + 1) : n_keys;
     if (prefix64 < 0) prefix64 = 0;
-    const int n = static_cast<int>(prefix64);
-    const int n_sel = n < k ? n : k;
-
-    if (tid == 0) { sh.n_cand = 0; sh.out_pos = 0; sh.eq_taken = 0; }
-    __syncthreads();
-
-    if (n <= k) {  // the whole prefix is selected
-        for (int i = tid; i < k; i += TK_THREADS) out[i] = i < n ? i : -1;
-        if (kth != nullptr || count != nullptr) {
-            float mn = __int_as_float(0x7f800000);
-            for (int i = tid; i < n; i += TK_THREADS) mn = fminf(mn, __ldcg(row + i));
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, d));
-            if (tid == 0) sh.red_lo = 0xffffffffu;
-            __syncthreads();
-            if ((tid & 31) == 0) atomicMin(&sh.red_lo, float_to_key(mn));
-            __syncthreads();
-            if (tid == 0) {
-                if (count) count[t] = n;
-                if (kth) kth[t] = n > 0 ? key_to_float(sh.red_lo) : __int_as_float(0xff800000);
-            }
-        }
-        return;
-    }
-
-    uint32_t thr = 0u;  // keep everything
-    const float4* row4 = reinterpret_cast<const float4*>(row);
-    if (n > TK_CAP) {
-        // ---- sample: thread i reads 8 consecutive floats at an evenly spread, 32-byte aligned offset
-        const int n8 = n >> 3;                       // complete 8-float groups
-        const int g = static_cast<int>((static_cast<int64_t>(tid) * (n8 - 1)) / (TK_THREADS - 1));
-        const float4 a = __ldcg(row4 + 2 * g), b = __ldcg(row4 + 2 * g + 1);
-        uint32_t* skey = sh.cand_key;                // the candidate buffer is free at this point
-        skey[tid * 8 + 0] = float_to_key(a.x); skey[tid * 8 + 1] = float_to_key(a.y);
-        skey[tid * 8 + 2] = float_to_key(a.z); skey[tid * 8 + 3] = float_to_key(a.w);
-        skey[tid * 8 + 4] = float_to_key(b.x); skey[tid * 8 + 5] = float_to_key(b.y);
-        skey[tid * 8 + 6] = float_to_key(b.z); skey[tid * 8 + 7] = float_to_key(b.w);
-        __syncthreads();
-        // rank in the sample whose value sits a few standard deviations below the true k-th
-        const float expect = static_cast<float>(TK_SAMPLE) * static_cast<float>(k) / static_cast<float>(n);
-        int r = static_cast<int>(expect + 4.0f * sqrtf(expect) + 8.0f);
-        if (r < TK_SAMPLE) {
-            int dummy;
-            SmemSource s{skey, nullptr, TK_SAMPLE};
-            thr = select_kth(s, r, sh, &dummy);
-        }
-        __syncthreads();
-    }
-
-    // ---- one streaming pass: keep elements at or above the threshold (a few per cent of the row)
-    {
-        const float thr_f = thr == 0u ? __int_as_float(0xff800000) : key_to_float(thr);
-        const int n4 = n >> 2;
-        constexpr int UNROLL = 4;                     // 16-byte loads in flight per thread
-        int i = tid;
-        for (; i + (UNROLL - 1) * TK_THREADS < n4; i += UNROLL * TK_THREADS) {
-            float4 x[UNROLL];
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) x[u] = __ldcs(row4 + i + u * TK_THREADS);
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const int e = 4 * (i + u * TK_THREADS);
-                keep_if_candidate(x[u].x, e, thr_f, sh);
-                keep_if_candidate(x[u].y, e + 1, thr_f, sh);
-                keep_if_candidate(x[u].z, e + 2, thr_f, sh);
-                keep_if_candidate(x[u].w, e + 3, thr_f, sh);
-            }
-        }
-        for (; i < n4; i += TK_THREADS) {
-            const float4 x = __ldcs(row4 + i);
-            keep_if_candidate(x.x, 4 * i, thr_f, sh);
-            keep_if_candidate(x.y, 4 * i + 1, thr_f, sh);
-            keep_if_candidate(x.z, 4 * i + 2, thr_f, sh);
-            keep_if_candidate(x.w, 4 * i + 3, thr_f, sh);
-        }
-        if (tid < n - 4 * n4) keep_if_candidate(__ldcg(row + 4 * n4 + tid), 4 * n4 + tid, thr_f, sh);   // ragged tail
-    }
-    __syncthreads();
-    const int n_cand = sh.n_cand;
-    uint32_t T;
-    int n_eq;
-    if (n_cand >= k && n_cand <= TK_CAP) {
-        SmemSource s{sh.cand_key, sh.cand_idx, n_cand};
-        T = select_kth(s, k, sh, &n_eq);
-        emit_selection(s, T, n_eq, out, sh);
-    } else {
-        GlobalSource s{row, n};
-        T = select_kth(s, k, sh, &n_eq);
-        emit_selection(s, T, n_eq, out, sh);
-    }
-    if (tid == 0) {
-        if (count) count[t] = n_sel;
-        if (kth) kth[t] = key_to_float(T);
-    }
+    topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix64), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh);
 }
 
 }  // namespace janus
