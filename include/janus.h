@@ -129,6 +129,42 @@ int janus_indexer_topk(const void* q_idx, int64_t q_stride_tok,
                        void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * janus_indexer_topk on scratch built into the library - no counterpart in the paper; a convenience of this library.
+ *
+ * Every other entry point takes its scratch from the caller.  This one is for callers that have none to give and cannot
+ * get any: code running inside a host program that has already handed all free device memory to its own KV-cache pool
+ * and lends none of it out, or a loop so latency-critical that it may not call the CUDA allocator (releasing device
+ * memory waits for the device to go idle).  The call allocates and frees nothing, on the host side of CUDA or through
+ * any library; its scratch is a fixed array of JANUS_STATIC_SCRATCH_BYTES in the library's device image, present once
+ * on every device that loads the library.
+ *
+ * Arguments, outputs and semantics are those of janus_indexer_topk without `ws` / `ws_bytes`.
+ *
+ *   Limit     janus_indexer_topk_workspace_size(...) for the same arguments must not exceed
+ *             JANUS_STATIC_SCRATCH_BYTES; otherwise the call returns JANUS_ERR_WORKSPACE_TOO_SMALL and touches
+ *             nothing.  64 MiB covers, for example, 128 new tokens over 131072 cached keys, or 64 over 262144
+ *             (64 x 128 FP8 indexer, k = 2048); a 4096-token chunk at that history needs the caller's workspace.
+ *   Set-up    the first call on a device looks up the array's address on that device (no allocation) and keeps it;
+ *             the device whose stream is passed must be the current device.  Make that first call before any
+ *             stream capture begins.
+ *   Sharing   all calls on one device use the same array.  Each call clears the counters it needs itself, so
+ *             nothing has to be zeroed beforehand and leftovers of earlier calls do not matter; but two calls that
+ *             may run at the same time (different streams, or different host threads without ordering between
+ *             their streams) race on it and give wrong results.  Order them on one stream or with events.
+ */
+#define JANUS_STATIC_SCRATCH_BYTES (64 << 20)
+int janus_indexer_topk_static(const void* q_idx, int64_t q_stride_tok,
+                              const void* k_idx, int64_t k_stride_tok,
+                              const float* w,
+                              const float* q_scale, int64_t q_scale_stride_tok,
+                              const float* k_scale,
+                              const float* row_bias, const float* col_bias,
+                              int M, int H_I, int D_I, int64_t n_keys,
+                              int64_t q_pos0, int causal, int dtype, int k,
+                              int32_t* idx, int32_t* count, float* kth,
+                              int32_t* dev_status, void* stream);
+
+/*
  * Page demand - union of the selections (Sec. 2.2), best-effort read packing into maximal runs of physically
  * adjacent pages (Sec. 4.3) and the corrective-read set "exact minus predicted" (Sec. 4.2).
  *

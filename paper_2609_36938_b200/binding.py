@@ -25,7 +25,7 @@ EXPORTS = [
     "janus_version", "janus_last_cuda_error",
     "janus_indexer_scores_workspace_size", "janus_indexer_scores",
     "janus_topk_workspace_size", "janus_topk",
-    "janus_indexer_topk_workspace_size", "janus_indexer_topk",
+    "janus_indexer_topk_workspace_size", "janus_indexer_topk", "janus_indexer_topk_static",
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
 ]
@@ -63,6 +63,9 @@ def load() -> ctypes.CDLL:
     lib.janus_indexer_topk.restype = c_i
     lib.janus_indexer_topk.argtypes = [c_p, c_i64, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i,
                                        c_p, c_p, c_p, c_p, c_sz, c_p, c_p]
+    lib.janus_indexer_topk_static.restype = c_i
+    lib.janus_indexer_topk_static.argtypes = [c_p, c_i64, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i,
+                                              c_p, c_p, c_p, c_p, c_p]
     lib.janus_page_demand_workspace_size.restype = c_sz
     lib.janus_page_demand_workspace_size.argtypes = [c_i64, c_i, c_i64]
     lib.janus_page_demand.restype = c_i
@@ -196,6 +199,32 @@ def janus_indexer_topk(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor
                                 _ptr(count), _ptr(kth), _ptr(workspace), workspace.numel(), _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_indexer_topk")
     return idx, count, kth
+
+
+STATIC_SCRATCH_BYTES = 64 << 20
+
+
+def janus_indexer_topk_static(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, k: int, idx: torch.Tensor, *,
+                              count: Optional[torch.Tensor] = None, kth: Optional[torch.Tensor] = None,
+                              q_scale: Optional[torch.Tensor] = None, k_scale: Optional[torch.Tensor] = None,
+                              row_bias: Optional[torch.Tensor] = None, col_bias: Optional[torch.Tensor] = None, q_pos0: int = 0,
+                              causal: bool = True) -> None:
+    """janus_indexer_topk on the scratch array built into the library.  Allocates nothing: the caller passes the outputs
+    (`idx` [M, k] int32, optionally `count` [M] int32 and `kth` [M] fp32).  Raises if the problem needs more scratch than
+    STATIC_SCRATCH_BYTES.  Calls on one device share the array: keep them ordered on the device."""
+    lib = load()
+    M, H, D = q_idx.shape
+    n_keys = k_idx.shape[0]
+    dtype = _idx_dtype_code(q_idx)
+    if _idx_dtype_code(k_idx) != dtype:
+        raise JanusError("q_idx and k_idx must share a dtype")
+    if idx.shape != (M, k) or idx.dtype != torch.int32 or not idx.is_contiguous():
+        raise JanusError("idx must be a contiguous [M, k] int32 tensor")
+    qs_stride = H if (q_scale is not None and q_scale.dim() == 2) else 0
+    rc = lib.janus_indexer_topk_static(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride,
+                                       _ptr(k_scale), _ptr(row_bias), _ptr(col_bias), M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype,
+                                       int(k), _ptr(idx), _ptr(count), _ptr(kth), _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_indexer_topk_static")
 
 
 def janus_page_demand(idx: torch.Tensor, *, demand_limit: int, page_size: int, page_table: torch.Tensor, n_phys_pages: int,

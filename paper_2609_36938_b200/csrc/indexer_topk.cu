@@ -11,6 +11,8 @@
 // Scratch (sample, thresholds, candidate lists, fallback rows) lives in the caller's workspace.
 // Shapes the tensor-core indexer does not take, and problems too small to sample, run the two-call path
 // (scores in the workspace, then the row-wise top-k).
+#include <mutex>
+
 #include "sm100_ptx.cuh"
 #include "topk_select.cuh"
 
@@ -349,4 +351,57 @@ extern "C" int janus_indexer_topk(const void* q_idx, int64_t q_stride_tok, const
     }
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
+}
+
+// ---- the same call on scratch that ships with the library ---------------------------------------------------------------------
+// Some callers have no device memory to hand over as a workspace and no way to get any: a plug-in running inside a serving
+// engine that has already given every free byte of HBM to its KV-cache pool and lends plug-ins none of it, or a
+// latency-critical loop that may not call the CUDA allocator because freeing device memory waits for the whole device.
+// For them the scratch is a fixed array in the library's own device image.  It exists once per device and is shared by every
+// call on that device.
+namespace janus {
+
+static __device__ __align__(256) unsigned char ft_static_scratch[JANUS_STATIC_SCRATCH_BYTES];
+
+// Device address of the array on the device that is current now, looked up the first time that device is seen.
+static int static_scratch_address(void** out) {
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex mu;
+    static void* address[MAX_DEVICES] = {};
+    int dev = -1;
+    JANUS_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return JANUS_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (address[dev] == nullptr) {
+        void* ptr = nullptr;
+        JANUS_CUDA_CHECK(cudaGetSymbolAddress((void**)&ptr, ft_static_scratch));
+        if (ptr == nullptr || !aligned16(ptr)) return JANUS_ERR_CUDA;
+        address[dev] = ptr;
+    }
+    *out = address[dev];
+    return JANUS_OK;
+}
+
+}  // namespace janus
+
+extern "C" int janus_indexer_topk_static(const void* q_idx, int64_t q_stride_tok, const void* k_idx, int64_t k_stride_tok, const float* w,
+                                         const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
+                                         const float* col_bias, int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal, int dtype,
+                                         int k, int32_t* idx, int32_t* count, float* kth, int32_t* dev_status, void* stream_) {
+    using namespace janus;
+    // the size check comes first: a problem that does not fit is refused before anything touches the device
+    if (M < 0 || H_I <= 0 || D_I <= 0 || n_keys < 0 || k <= 0) return JANUS_ERR_INVALID_ARG;
+    if (M > 0 && n_keys > 0) {
+        const FusedLayout L = fused_layout(M, H_I, D_I, n_keys, q_pos0, causal, dtype, k);
+        size_t need = L.total;
+        if (L.fused && q_stride_tok != static_cast<int64_t>(H_I) * D_I)   // strided queries take the two-call route
+            need = align_up(sizeof(float) * static_cast<size_t>(L.ld) * M);
+        if (need > static_cast<size_t>(JANUS_STATIC_SCRATCH_BYTES)) return JANUS_ERR_WORKSPACE_TOO_SMALL;
+    }
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != JANUS_OK) return rc;
+    return janus_indexer_topk(q_idx, q_stride_tok, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias, M, H_I, D_I,
+                              n_keys, q_pos0, causal, dtype, k, idx, count, kth, scratch, static_cast<size_t>(JANUS_STATIC_SCRATCH_BYTES), dev_status,
+                              stream_);
 }
