@@ -24,8 +24,11 @@
 //   warps 1-6    gather: each owns one ring slot, resolves its 32 rows through the page table (one half-tile ahead)
 //                and copies this CTA's bytes with 16-byte cp.async into the 128-byte-swizzled K-major layout;
 //   warps 7-10   exchange: as soon as a partial logit tile is complete they send it to the peer, so the transfer of
-//                tile i+1 overlaps the softmax of tile i;
+//                tile i+1 overlaps the softmax of tile i; after a token's last tile they load the next token's queries;
 //   warps 11-14  softmax (thread = head): add the peer's partial logits, fp32 online softmax, write P (bf16) over the logits.
+// The kernel is persistent: one cluster per SM pair loops over tokens, and the ring, the logit buffers and all barrier
+// phases run on across tokens, so a token's prologue (queries into tensor memory, first gathers) hides behind the previous
+// token's last tiles and output.
 // The running max only moves when a tile exceeds it by more than 2^8, so O is rescaled (in TMEM) a handful of times
 // per row.  Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT, and both CTAs of the cluster
 // still meet at the final cluster barrier.
@@ -90,7 +93,7 @@ struct LpParams {
 #define LP_PROF_WAIT(acc, expr) ([&] { const long long _t0 = clock64(); const bool _r = (expr); acc += clock64() - _t0; return _r; }())
 #define LP_PROF_NOW() clock64()
 #define LP_PROF_SEG(acc, t_prev) do { const long long _n = clock64(); acc += _n - t_prev; t_prev = _n; } while (0)
-#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == 0u) p.lse[static_cast<int64_t>(t) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
+#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == 0u) p.lse[static_cast<int64_t>(cid) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
 #else
 #define LP_PROF_DECL(name)
 #define LP_PROF_WAIT(acc, expr) (expr)
@@ -120,7 +123,11 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t c = cluster_ctarank();          // 0 or 1: which bytes of the rows this CTA owns
     const uint32_t peer = c ^ 1u;
-    const int t = blockIdx.x >> 1;
+    // persistent: cluster `cid` handles tokens cid, cid + n_clusters, ...; the key ring, the logit buffers and every barrier
+    // phase run on across tokens (tiles are counted globally), so the next token's rows are gathered, and its queries
+    // loaded, while the current token's last tiles and output are still in flight
+    const int cid = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    const int n_my = cid < p.M ? (p.M - cid + n_clusters - 1) / n_clusters : 0;
     const int n_atoms = 4 + static_cast<int>(c);
     const int n_tiles = (p.k + LP_TILE - 1) / LP_TILE;
     const int n_half = 2 * n_tiles;
@@ -163,69 +170,77 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         // ================================================================== MMA issue (whole warp runs the loop, lane 0 issues)
         const bool leader = lane == 0;
         const uint32_t qf = smem_u32(&sh->q_full);
-        if (leader) {
+        auto fetch_q4 = [&](int it) {      // rope dims [512,576) of all heads of this cluster's token `it` (CTA 1 only)
+            if (!leader) return;
             if (c == 1u) {
                 mbar_expect_tx(qf, LP_Q_ATOM_BYTES);
-                tma_load_2d(smem_u32(q4_smem), &tmap_q, 512, t * LP_HEADS, qf);     // rope dims [512,576) of all heads
+                tma_load_2d(smem_u32(q4_smem), &tmap_q, 512, (cid + it * n_clusters) * LP_HEADS, qf);
             } else {
                 mbar_arrive(qf);
             }
-        }
+        };
+        if (n_my > 0) fetch_q4(0);
         constexpr uint32_t idesc_qk = umma_idesc_major(1u, LP_HEADS, LP_TILE, 0u, 0u);
         constexpr uint32_t idesc_pv = umma_idesc_major(1u, LP_HEADS, LP_DVH, 0u, 1u);
         LP_PROF_DECL(w_kfull); LP_PROF_DECL(w_pfull); LP_PROF_DECL(w_q);
         const long long prof_t0 = LP_PROF_NOW();
-        bool ok = LP_PROF_WAIT(w_q, mbar_wait(qf, 0) && mbar_wait(smem_u32(&sh->qt_full), 0));
-        tc_fence_after();
         const uint32_t q4_lo = umma_desc_lo(smem_u32(q4_smem), 16);
         const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem), 16);
         const uint32_t v_lo = umma_desc_lo(smem_u32(k_smem), LP_K_ATOM_BYTES);     // value half = first four owned atoms
-        auto issue_pv = [&](int j) {   // O += P_j . V_j
+        auto issue_pv = [&](int j, bool first) {   // O += P_j . V_j (j counts tiles globally; `first`: the token's first tile)
             const int b = j & 1, buf = j % LP_BUFS;
             const uint32_t vb = v_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
             const uint32_t pa = tmem_base + LP_COL_S + b * LP_TILE;
             if (leader) {
 #pragma unroll
                 for (int ks = 0; ks < LP_TILE / 16; ++ks)
-                    umma_bf16_ts_lohi(tmem_base + LP_COL_O, pa + ks * 8, vb + ks * (2048 >> 4), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    umma_bf16_ts_lohi(tmem_base + LP_COL_O, pa + ks * 8, vb + ks * (2048 >> 4), idesc_pv, (!first || ks > 0) ? 1u : 0u);
                 umma_commit(smem_u32(&sh->k_empty[buf]));   // tile buffer free again, and "P.V of tile j done" for the softmax warps
             }
         };
-        for (int i = 0; i < n_tiles && ok; ++i) {
-            const int b = i & 1, buf = i % LP_BUFS;
-            ok = LP_PROF_WAIT(w_kfull, mbar_wait(smem_u32(&sh->k_full[buf]), static_cast<uint32_t>(i / LP_BUFS) & 1u));
+        bool ok = true;
+        int gi = 0;                                  // tiles issued so far, over all tokens
+        for (int it = 0; it < n_my && ok; ++it) {
+            ok = LP_PROF_WAIT(w_q, mbar_wait(qf, static_cast<uint32_t>(it) & 1u) && mbar_wait(smem_u32(&sh->qt_full), static_cast<uint32_t>(it) & 1u));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_s = tmem_base + LP_COL_S + b * LP_TILE;
-            const uint32_t kb = k_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
-            if (leader) {
-#pragma unroll
-                for (int a = 0; a < 4; ++a) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_bf16_ts_lohi(d_s, tmem_base + LP_COL_Q + a * 32 + ks * 8, kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk,
-                                          (a > 0 || ks > 0) ? 1u : 0u);
-                }
-                if (c == 1u) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_bf16_ss_lohi(d_s, q4_lo + ks * 2, kb + 4 * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk, 1u);
-                }
-                umma_commit(smem_u32(&sh->s_full[b]));
-            }
-            if (i >= 1) {
-                ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(i - 1) & 1]), static_cast<uint32_t>((i - 1) >> 1) & 1u));
+            for (int i = 0; i < n_tiles; ++i, ++gi) {
+                const int b = gi & 1, buf = gi % LP_BUFS;
+                ok = LP_PROF_WAIT(w_kfull, mbar_wait(smem_u32(&sh->k_full[buf]), static_cast<uint32_t>(gi / LP_BUFS) & 1u));
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(i - 1);
+                const uint32_t d_s = tmem_base + LP_COL_S + b * LP_TILE;
+                const uint32_t kb = k_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
+                if (leader) {
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16_ts_lohi(d_s, tmem_base + LP_COL_Q + a * 32 + ks * 8, kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk,
+                                              (a > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    if (c == 1u) {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16_ss_lohi(d_s, q4_lo + ks * 2, kb + 4 * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk, 1u);
+                    }
+                    umma_commit(smem_u32(&sh->s_full[b]));
+                }
+                if (i >= 1) {
+                    ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(gi - 1) & 1]), static_cast<uint32_t>((gi - 1) >> 1) & 1u));
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(gi - 1, i == 1);
+                }
             }
-        }
-        if (ok && n_tiles > 0) {
-            ok = mbar_wait(smem_u32(&sh->p_full[(n_tiles - 1) & 1]), static_cast<uint32_t>((n_tiles - 1) >> 1) & 1u);
-            if (ok) {
-                tc_fence_after();
-                issue_pv(n_tiles - 1);
-            }
+            if (!ok) break;
+            // the token's last P: once it exists, every logit MMA of the token has completed, so the queries may be replaced;
+            // the output of the token has been read out of O before the softmax warps produce the next token's first P
+            ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(gi - 1) & 1]), static_cast<uint32_t>((gi - 1) >> 1) & 1u));
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(gi - 1, n_tiles == 1);
+            if (it + 1 < n_my) fetch_q4(it + 1);
         }
         if (!ok && leader) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
         if (leader) { LP_PROF_PUT(0, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(1, w_kfull); LP_PROF_PUT(2, w_pfull); LP_PROF_PUT(9, w_q); }
@@ -235,15 +250,17 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         // half-tile and no two warps ever synchronise.  Because every use of a slot is made by the same warp, the slot's
         // barrier is at most one phase ahead of it, which the parity wait relies on.
         const int g = warp - 1;
-        const int32_t* my_idx = p.idx + static_cast<int64_t>(t) * p.k;
+        const int total_half = n_my * n_half;                  // half-tiles of all tokens of this cluster, counted globally
         const int n_chunks = 8 * n_atoms;                      // 16-byte chunks of a row owned by this CTA (32 or 40)
         const int64_t seg_off = 512 * static_cast<int64_t>(c); // first owned byte of a row
         bool ok = true;
         LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
         const long long prof_t0 = LP_PROF_NOW();
-        auto load_raw = [&](int hi) -> int {                   // lane r owns row r of half-tile hi
-            const int slot = hi * LP_HALF + lane;
-            return (hi < n_half && slot < p.k) ? __ldg(my_idx + slot) : -1;
+        auto load_raw = [&](int gh) -> int {                   // lane r owns row r of global half-tile gh
+            if (gh >= total_half) return -1;
+            const int it = gh / n_half;
+            const int slot = (gh - it * n_half) * LP_HALF + lane;
+            return slot < p.k ? __ldg(p.idx + static_cast<int64_t>(cid + it * n_clusters) * p.k + slot) : -1;
         };
         auto resolve = [&](int s_tok, bool& valid) -> const unsigned char* {   // first owned byte of the row of token s_tok
             const unsigned char* ptr = reinterpret_cast<const unsigned char*>(p.pool) + seg_off;
@@ -265,7 +282,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const unsigned char* row_ptr = resolve(load_raw(g), valid_cur);
         const unsigned char* row_nxt = row_ptr;
         int raw_nxt = load_raw(g + LP_GATHER_WARPS);
-        for (int hi = g; hi < n_half; hi += LP_GATHER_WARPS) {
+        for (int hi = g; hi < total_half; hi += LP_GATHER_WARPS) {
             const int buf = (hi >> 1) % LP_BUFS, hf = hi & 1;
             const bool s_ok = valid_cur;
             const uint32_t valid_mask = __ballot_sync(0xffffffffu, s_ok);
@@ -309,10 +326,30 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const uint32_t peer_xbuf = mapa_shared(smem_u32(xbuf), peer);
         const uint32_t peer_xfull = mapa_shared(smem_u32(&sh->x_full[0]), peer);
+        // this CTA's first 256 query dims of head h of the cluster's token `it` -> tensor memory, two bf16 per 32-bit column
+        auto load_q = [&](int it) {
+            const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(cid + it * n_clusters) * LP_HEADS + h) * LP_DQK + 256 * c);
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                uint32_t r[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint4 u = __ldg(src + a * 8 + v);
+                    r[4 * v + 0] = u.x; r[4 * v + 1] = u.y; r[4 * v + 2] = u.z; r[4 * v + 3] = u.w;
+                }
+                tmem_st32_wait(lane_addr + LP_COL_Q + a * 32, r);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->qt_full));
+        };
+        if (n_my > 0) load_q(0);
         bool ok = true;
-        for (int i = 0; i < n_tiles; ++i) {
-            const int b = i & 1;
-            const uint32_t ph = static_cast<uint32_t>(i >> 1) & 1u;
+        int gi = 0;
+        for (int it = 0; it < n_my && ok; ++it) {
+        for (int i = 0; i < n_tiles; ++i, ++gi) {
+            const int b = gi & 1;
+            const uint32_t ph = static_cast<uint32_t>(gi >> 1) & 1u;
             // the logits are complete, and the peer has read what this CTA sent two tiles ago into the same buffer
             ok = mbar_wait(smem_u32(&sh->s_full[b]), ph) && mbar_wait(smem_u32(&sh->x_empty[b]), ph ^ 1u);
             ok = __all_sync(0xffffffffu, ok);
@@ -338,32 +375,16 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                                            __uint_as_float(r[4 * j4 + 1]), __uint_as_float(r[4 * j4 + 2]), __uint_as_float(r[4 * j4 + 3]), bar);
             }
         }
+            // the token's last logit tile is complete, so nothing reads its queries any more: bring in the next token's
+            if (ok && it + 1 < n_my) load_q(it + 1);
+        }
         if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
     } else {
         // ================================================================== softmax + output: 4 warps, thread = head
         const int quad = warp & 3;
         const int h = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-        // this CTA's first 256 query dims of this head -> tensor memory, two bf16 per 32-bit column
-        {
-            const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DQK + 256 * c);
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                uint32_t r[32];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const uint4 u = __ldg(src + a * 8 + v);
-                    r[4 * v + 0] = u.x; r[4 * v + 1] = u.y; r[4 * v + 2] = u.z; r[4 * v + 3] = u.w;
-                }
-                tmem_st32_wait(lane_addr + LP_COL_Q + a * 32, r);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->qt_full));
-        }
         const float neg_inf = __int_as_float(0xff800000);
-        float m_ref = neg_inf;      // reference maximum (scaled, log2 domain) the exponentials are taken against
-        float l_sum = 0.f;
         bool ok = true;
         LP_PROF_DECL(w_sfull); LP_PROF_DECL(w_xfull); LP_PROF_DECL(w_send);
         LP_PROF_DECL(s_ld); LP_PROF_DECL(s_peer); LP_PROF_DECL(s_arr); LP_PROF_DECL(s_exp); LP_PROF_DECL(s_st);
@@ -371,9 +392,14 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         long long seg = prof_t0;
         (void)seg;
         const uint32_t peer_xempty = mapa_shared(smem_u32(&sh->x_empty[0]), peer);
-        for (int i = 0; i < n_tiles; ++i) {
-            const int b = i & 1, buf = i % LP_BUFS;
-            const uint32_t ph_k = static_cast<uint32_t>(i / LP_BUFS) & 1u, ph_s = static_cast<uint32_t>(i >> 1) & 1u;
+        int gi = 0;                 // tiles done so far, over all tokens
+        for (int it = 0; it < n_my && ok; ++it) {
+        const int t = cid + it * n_clusters;
+        float m_ref = neg_inf;      // reference maximum (scaled, log2 domain) the exponentials are taken against
+        float l_sum = 0.f;
+        for (int i = 0; i < n_tiles; ++i, ++gi) {
+            const int b = gi & 1, buf = gi % LP_BUFS;
+            const uint32_t ph_k = static_cast<uint32_t>(gi / LP_BUFS) & 1u, ph_s = static_cast<uint32_t>(gi >> 1) & 1u;
             // this CTA's exchange barrier for the tile: expect the peer's 32 KB of partial logits
             if (warp == LP_SMAX_WARP0 && lane == 0) mbar_expect_tx(smem_u32(&sh->x_full[b]), LP_XBUF_BYTES);
             // k_full is complete long before s_full; waiting on it as well makes the validity masks written by the gather
@@ -434,7 +460,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             }
             if (__any_sync(0xffffffffu, moved) && i > 0) {
                 // rescale O in tensor memory: the previous tile's P.V must have completed first
-                ok = mbar_wait(smem_u32(&sh->k_empty[(i - 1) % LP_BUFS]), static_cast<uint32_t>((i - 1) / LP_BUFS) & 1u);
+                ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -471,45 +497,45 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (lane == 0) mbar_arrive(smem_u32(&sh->p_full[b]));
             LP_PROF_SEG(s_st, seg);
         }
-        // ---- output: wait for the last P.V, normalise, round to bf16
-        if (ok && n_tiles > 0) {
-            ok = mbar_wait(smem_u32(&sh->k_empty[(n_tiles - 1) % LP_BUFS]), static_cast<uint32_t>((n_tiles - 1) / LP_BUFS) & 1u);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok) {
-            tc_fence_after();
-            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            const bool have_o = n_tiles > 0 && __any_sync(0xffffffffu, l_sum > 0.f);   // some P.V has written O
-            uint16_t* orow = p.out + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DV + c * LP_DVH;
+        if (!ok) break;
+        // ---- output: wait for the token's last P.V, normalise, round to bf16.  The next token's first P is produced by
+        // these same warps afterwards, so its P.V cannot overwrite O before O has been read here.
+        ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+        const bool have_o = __any_sync(0xffffffffu, l_sum > 0.f);   // some P.V of this token has written O
+        uint16_t* orow = p.out + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DV + c * LP_DVH;
 #pragma unroll 1
-            for (int cc = 0; cc < LP_DVH / 32; ++cc) {
-                uint32_t o[32];
-                if (have_o) {
-                    tmem_ld32_wait(lane_addr + LP_COL_O + cc * 32, o);
-                } else {
+        for (int cc = 0; cc < LP_DVH / 32; ++cc) {
+            uint32_t o[32];
+            if (have_o) {
+                tmem_ld32_wait(lane_addr + LP_COL_O + cc * 32, o);
+            } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) o[j] = 0u;
-                }
-                uint4* dst = reinterpret_cast<uint4*>(orow + cc * 32);
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint4 u;
-                    u.x = lp_pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                    u.y = lp_pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                    u.z = lp_pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                    u.w = lp_pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                    dst[v] = u;
-                }
+                for (int j = 0; j < 32; ++j) o[j] = 0u;
             }
-#ifndef JANUS_ATTN_PROFILE
-            if (p.lse != nullptr && c == 0u)
-                p.lse[static_cast<int64_t>(t) * LP_HEADS + h] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : neg_inf;
-#else
-            if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); }
-#endif
-        } else if (lane == 0) {
-            report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+            uint4* dst = reinterpret_cast<uint4*>(orow + cc * 32);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                uint4 u;
+                u.x = lp_pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                u.y = lp_pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                u.z = lp_pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                u.w = lp_pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                dst[v] = u;
+            }
         }
+#ifndef JANUS_ATTN_PROFILE
+        if (p.lse != nullptr && c == 0u)
+            p.lse[static_cast<int64_t>(t) * LP_HEADS + h] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : neg_inf;
+#endif
+        }
+        if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+#ifdef JANUS_ATTN_PROFILE
+        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); }
+#endif
     }
     tc_fence_before();
     __syncthreads();
@@ -556,7 +582,34 @@ int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t
         return JANUS_ERR_CUDA;
     const size_t smem = LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES + LP_Q_ATOM_BYTES + sizeof(LpShared) + 16;
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(sparse_attn_latent_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    sparse_attn_latent_pair_kernel<<<2 * M, LP_THREADS, smem, stream>>>(tq, p);   // clusters of 2 CTAs (compile-time cluster dims)
+    // persistent launch: as many 2-CTA clusters as the device keeps resident at once (one CTA per SM), each looping over tokens
+    static int resident_clusters[64] = {};
+    int dev = 0;
+    JANUS_CUDA_CHECK(cudaGetDevice(&dev));
+    int n_clusters = (dev >= 0 && dev < 64) ? resident_clusters[dev] : 0;
+    if (n_clusters <= 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 148);
+        cfg.blockDim = dim3(LP_THREADS);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, sparse_attn_latent_pair_kernel, &cfg) != cudaSuccess || n_clusters <= 0) {
+            (void)cudaGetLastError();
+            int sms = 0;
+            JANUS_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+            n_clusters = sms / 2;
+        }
+        if (n_clusters <= 0) n_clusters = 1;
+        if (dev >= 0 && dev < 64) resident_clusters[dev] = n_clusters;
+    }
+    if (n_clusters > M) n_clusters = M;
+    sparse_attn_latent_pair_kernel<<<2 * n_clusters, LP_THREADS, smem, stream>>>(tq, p);   // clusters of 2 CTAs (compile-time cluster dims)
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
