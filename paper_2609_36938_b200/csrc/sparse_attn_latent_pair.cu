@@ -251,7 +251,8 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         // barrier is at most one phase ahead of it, which the parity wait relies on.
         const int g = warp - 1;
         const int total_half = n_my * n_half;                  // half-tiles of all tokens of this cluster, counted globally
-        const int n_chunks = 8 * n_atoms;                      // 16-byte chunks of a row owned by this CTA (32 or 40)
+        const int g_sub = lane & 3, g_rr = lane >> 2;          // this lane copies piece g_sub of the 64-byte groups of rows 8q + g_rr
+        const uint32_t g_sw0 = static_cast<uint32_t>((g_sub ^ g_rr) << 4), g_sw1 = static_cast<uint32_t>(((4 + g_sub) ^ g_rr) << 4);
         const int64_t seg_off = 512 * static_cast<int64_t>(c); // first owned byte of a row
         bool ok = true;
         LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
@@ -292,20 +293,23 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (!ok) break;
             if (lane == 0) sh->vmask[2 * buf + hf] = valid_mask;
             const uint32_t stage_base = smem_u32(k_smem + buf * LP_TILE_BYTES + hf * LP_HALF * 128);
-            // lane l copies 16-byte chunk l (and chunk 32+l of a 640-byte segment) of every row: chunk ch of the owned bytes
-            // goes to atom ch/8, position (ch%8) ^ (r%8) inside the 128-byte row r
-            const uint32_t dst0 = stage_base + (lane >> 3) * LP_K_ATOM_BYTES + ((lane & 7) << 4);
-            const uint32_t dst1 = dst0 + 4 * LP_K_ATOM_BYTES;
-            const bool second = lane + 32 < n_chunks;
+            // One instruction copies 64 contiguous bytes (4 lanes x 16) of each of 8 rows, so a row pointer is fetched from
+            // its owner lane once per 8 rows and every copy is a single instruction with immediate offsets: chunk ch of the
+            // owned bytes goes to atom ch/8, position (ch%8) ^ (r%8) inside the 128-byte row r.
             const uint32_t lo = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr)), hi32 = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr) >> 32);
-#pragma unroll 8
-            for (int r = 0; r < LP_HALF; ++r) {
+#pragma unroll
+            for (int q = 0; q < LP_HALF / 8; ++q) {
+                const int r = 8 * q + g_rr;
                 const uint64_t pr = (static_cast<uint64_t>(__shfl_sync(0xffffffffu, hi32, r)) << 32) | __shfl_sync(0xffffffffu, lo, r);
-                const unsigned char* src = reinterpret_cast<const unsigned char*>(pr) + lane * 16;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(pr) + g_sub * 16;
                 const uint32_t bytes = ((valid_mask >> r) & 1u) ? 16u : 0u;
-                const uint32_t swz = static_cast<uint32_t>((r & 7) << 4);
-                cp_async16((dst0 ^ swz) + r * 128, src, bytes);
-                if (second) cp_async16((dst1 ^ swz) + r * 128, src + 512, bytes);
+                const uint32_t d = stage_base + static_cast<uint32_t>(r * 128);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cp_async16(d + (i >> 1) * LP_K_ATOM_BYTES + ((i & 1) ? g_sw1 : g_sw0), src + i * 64, bytes);
+                if (c == 1u) {
+                    cp_async16(d + 4 * LP_K_ATOM_BYTES + g_sw0, src + 512, bytes);
+                    cp_async16(d + 4 * LP_K_ATOM_BYTES + g_sw1, src + 576, bytes);
+                }
             }
             cp_async_commit();
             row_nxt = resolve(raw_nxt, valid_nxt);                 // page-table load overlaps the copies in flight
@@ -409,14 +413,14 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (!ok) break;
             tc_fence_after();
             const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
-            float x[LP_TILE];
+            float2 x[LP_TILE / 2];          // logits of keys 2j, 2j+1
             seg = LP_PROF_NOW();
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t r[32];
                 tmem_ld32_wait(s_addr + hf * 32, r);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) x[hf * 32 + j] = __uint_as_float(r[j]);
+                for (int j = 0; j < 16; ++j) x[hf * 16 + j] = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
             }
             LP_PROF_SEG(s_ld, seg);
             // the peer's partial logits of the same tile (bytes counted as they land: visible once the phase completes)
@@ -430,18 +434,26 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
 #pragma unroll
                 for (int j4 = 0; j4 < LP_TILE / 4; ++j4) {
                     const float4 pv = xin[j4 * LP_HEADS];
-                    x[4 * j4 + 0] += pv.x; x[4 * j4 + 1] += pv.y; x[4 * j4 + 2] += pv.z; x[4 * j4 + 3] += pv.w;
+                    x[2 * j4] = fadd2(x[2 * j4], make_float2(pv.x, pv.y));
+                    x[2 * j4 + 1] = fadd2(x[2 * j4 + 1], make_float2(pv.z, pv.w));
                 }
                 const uint32_t vm0 = sh->vmask[2 * buf], vm1 = sh->vmask[2 * buf + 1];
                 if ((vm0 & vm1) != 0xffffffffu) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        x[j] = ((vm0 >> j) & 1u) ? x[j] : neg_inf;
-                        x[32 + j] = ((vm1 >> j) & 1u) ? x[32 + j] : neg_inf;
+                    for (int j = 0; j < 16; ++j) {
+                        x[j].x = ((vm0 >> (2 * j)) & 1u) ? x[j].x : neg_inf;
+                        x[j].y = ((vm0 >> (2 * j + 1)) & 1u) ? x[j].y : neg_inf;
+                        x[16 + j].x = ((vm1 >> (2 * j)) & 1u) ? x[16 + j].x : neg_inf;
+                        x[16 + j].y = ((vm1 >> (2 * j + 1)) & 1u) ? x[16 + j].y : neg_inf;
                     }
                 }
+                float mx[4] = {neg_inf, neg_inf, neg_inf, neg_inf};
 #pragma unroll
-                for (int j = 0; j < LP_TILE; ++j) tile_max = fmaxf(tile_max, x[j]);
+                for (int j = 0; j < LP_TILE / 2; j += 4) {
+                    mx[0] = fmax3(mx[0], x[j].x, x[j].y); mx[1] = fmax3(mx[1], x[j + 1].x, x[j + 1].y);
+                    mx[2] = fmax3(mx[2], x[j + 2].x, x[j + 2].y); mx[3] = fmax3(mx[3], x[j + 3].x, x[j + 3].y);
+                }
+                tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             }
             LP_PROF_SEG(s_peer, seg);
             // the exchange buffer has been read: the peer may send the tile after next into it
@@ -474,17 +486,20 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                 }
             }
             const float neg_m = (m_ref == neg_inf) ? 0.f : -m_ref;
-            // P is cut (not rounded) to bf16 with integer ops, which keeps the conversion off the quarter-rate unit the
-            // exponentials already occupy; the row sum adds the very same cut values, so the normalisation stays consistent
+            // P is rounded to bf16 (one pack instruction per pair); the row sum adds the very same rounded values, so the
+            // normalisation stays consistent and the log-sum-exp is not biased
             uint32_t pk[32];
-            float tile_sum = 0.f;
+            float2 ts[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            const float2 sc2 = make_float2(p.scale_log2e, p.scale_log2e), nm2 = make_float2(neg_m, neg_m);
 #pragma unroll
             for (int j = 0; j < LP_TILE / 2; ++j) {
-                const uint32_t u0 = __float_as_uint(lp_exp2(fmaf(x[2 * j], p.scale_log2e, neg_m))) & 0xffff0000u;
-                const uint32_t u1 = __float_as_uint(lp_exp2(fmaf(x[2 * j + 1], p.scale_log2e, neg_m))) & 0xffff0000u;
-                tile_sum += __uint_as_float(u0) + __uint_as_float(u1);
-                pk[j] = __byte_perm(u0, u1, 0x7632);       // low half = bf16(p0), high half = bf16(p1)
+                const float2 e = ffma2(x[j], sc2, nm2);
+                pk[j] = lp_pack_bf16x2(lp_exp2(e.x), lp_exp2(e.y));       // low half = bf16(p of key 2j), high half = bf16(p of key 2j+1)
+                ts[j & 3] = fadd2(ts[j & 3], make_float2(__uint_as_float(pk[j] << 16), __uint_as_float(pk[j] & 0xffff0000u)));
             }
+            const float2 t01 = fadd2(ts[0], ts[1]), t23 = fadd2(ts[2], ts[3]);
+            const float2 t4 = fadd2(t01, t23);
+            const float tile_sum = t4.x + t4.y;
             l_sum += tile_sum;
             LP_PROF_SEG(s_exp, seg);
             // P overwrites the first 32 columns of the logits: the exchange warps must have read them
