@@ -93,7 +93,10 @@ struct LpParams {
 #define LP_PROF_WAIT(acc, expr) ([&] { const long long _t0 = clock64(); const bool _r = (expr); acc += clock64() - _t0; return _r; }())
 #define LP_PROF_NOW() clock64()
 #define LP_PROF_SEG(acc, t_prev) do { const long long _n = clock64(); acc += _n - t_prev; t_prev = _n; } while (0)
-#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == 0u) p.lse[static_cast<int64_t>(cid) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
+#ifndef JANUS_PROF_CTA
+#define JANUS_PROF_CTA 0u
+#endif
+#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == JANUS_PROF_CTA) p.lse[static_cast<int64_t>(cid) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
 #else
 #define LP_PROF_DECL(name)
 #define LP_PROF_WAIT(acc, expr) (expr)
@@ -351,6 +354,13 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         bool ok = true;
         int gi = 0;
         for (int it = 0; it < n_my && ok; ++it) {
+        if (it + 1 < n_my) {
+            // the next token's queries are wanted the moment this token's last logit tile is done: have them in L2 by then
+            const unsigned char* nq = reinterpret_cast<const unsigned char*>(p.q + (static_cast<int64_t>(cid + (it + 1) * n_clusters) * LP_HEADS + h) * LP_DQK + 256 * c);
+#pragma unroll
+            for (int a = 0; a < 4; ++a) prefetch_l2(nq + a * 128);
+            prefetch_l2(nq + 496);
+        }
         for (int i = 0; i < n_tiles; ++i, ++gi) {
             const int b = gi & 1;
             const uint32_t ph = static_cast<uint32_t>(gi >> 1) & 1u;
@@ -389,8 +399,10 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const int h = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const float neg_inf = __int_as_float(0xff800000);
+        const bool out_al32 = (reinterpret_cast<uint64_t>(p.out) & 31u) == 0u;
         bool ok = true;
         LP_PROF_DECL(w_sfull); LP_PROF_DECL(w_xfull); LP_PROF_DECL(w_send);
+        LP_PROF_DECL(e_wait); LP_PROF_DECL(e_out);
         LP_PROF_DECL(s_ld); LP_PROF_DECL(s_peer); LP_PROF_DECL(s_arr); LP_PROF_DECL(s_exp); LP_PROF_DECL(s_st);
         const long long prof_t0 = LP_PROF_NOW();
         long long seg = prof_t0;
@@ -513,12 +525,14 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             LP_PROF_SEG(s_st, seg);
         }
         if (!ok) break;
+        seg = LP_PROF_NOW();
         // ---- output: wait for the token's last P.V, normalise, round to bf16.  The next token's first P is produced by
         // these same warps afterwards, so its P.V cannot overwrite O before O has been read here.
         ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
+        LP_PROF_SEG(e_wait, seg);
         const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
         const bool have_o = __any_sync(0xffffffffu, l_sum > 0.f);   // some P.V of this token has written O
         uint16_t* orow = p.out + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DV + c * LP_DVH;
@@ -531,17 +545,19 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
 #pragma unroll
                 for (int j = 0; j < 32; ++j) o[j] = 0u;
             }
-            uint4* dst = reinterpret_cast<uint4*>(orow + cc * 32);
+            uint32_t w[16];
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                uint4 u;
-                u.x = lp_pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                u.y = lp_pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                u.z = lp_pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                u.w = lp_pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                dst[v] = u;
+            for (int j = 0; j < 16; ++j) w[j] = lp_pack_bf16x2(__uint_as_float(o[2 * j]) * inv, __uint_as_float(o[2 * j + 1]) * inv);
+            if (out_al32) {      // whole 32-byte sectors per thread: half the store instructions and transactions
+                st_global_v8(orow + cc * 32, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                st_global_v8(orow + cc * 32 + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(orow + cc * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
             }
         }
+        LP_PROF_SEG(e_out, seg);
 #ifndef JANUS_ATTN_PROFILE
         if (p.lse != nullptr && c == 0u)
             p.lse[static_cast<int64_t>(t) * LP_HEADS + h] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : neg_inf;
@@ -549,7 +565,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         }
         if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
 #ifdef JANUS_ATTN_PROFILE
-        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); }
+        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); LP_PROF_PUT(16, e_wait); LP_PROF_PUT(17, e_out); }
 #endif
     }
     tc_fence_before();
