@@ -47,7 +47,8 @@ constexpr int LP_HALF = 32;                 // rows per half-tile (gather / ring
 constexpr int LP_TILE = 2 * LP_HALF;        // keys per MMA tile
 constexpr int LP_BUFS = 3;                  // 64-key tile buffers
 constexpr int LP_SLOTS = 2 * LP_BUFS;       // ring slots (half-tiles)
-constexpr int LP_GATHER_WARPS = 6;          // one per ring slot (must divide LP_SLOTS)
+constexpr int LP_GATHER_WARPS = 3;          // warp g owns ring slots g and g + 3 (must divide LP_SLOTS); 12 warps in all leave
+                                            // 168 registers per thread, which the softmax needs to stay out of local memory
 constexpr int LP_ATOMS_MAX = 5;             // 64-dim atoms owned by a CTA: 4 (CTA 0) or 5 (CTA 1)
 constexpr int LP_K_ATOM_BYTES = LP_TILE * 128;                   // 8 KB
 constexpr int LP_TILE_BYTES = LP_ATOMS_MAX * LP_K_ATOM_BYTES;    // 40 KB
@@ -55,7 +56,7 @@ constexpr int LP_XBUF_BYTES = LP_TILE * LP_HEADS * 4;            // 32 KB: parti
 constexpr int LP_Q_ATOM_BYTES = LP_HEADS * 128;                  // 16 KB
 constexpr int LP_XCHG_WARP0 = 1 + LP_GATHER_WARPS;               // first exchange warp
 constexpr int LP_SMAX_WARP0 = LP_XCHG_WARP0 + 4;                 // first softmax warp
-constexpr int LP_THREADS = 32 * (LP_SMAX_WARP0 + 4);             // 15 warps
+constexpr int LP_THREADS = 32 * (LP_SMAX_WARP0 + 4);             // 12 warps
 constexpr uint32_t LP_COL_O = 0, LP_COL_S = 256, LP_COL_Q = 384;
 
 struct LpShared {
