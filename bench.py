@@ -43,13 +43,14 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.rows = []
+        self.skip = 0
         self.proc = None
 
     def start(self):
         q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.index)],
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "25", "-i", str(self.index)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -59,6 +60,17 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
+
+    def wait_until_running(self, timeout_s: float = 10.0):
+        """Blocks until nvidia-smi has delivered its first sample, then forgets the samples taken so far: its start-up
+        (driver initialisation on every GPU of the box) otherwise falls into the warm-up or timed steps and shows up as a
+        multi-millisecond gap inside whichever kernel is running, and an idle sample is not a sample under load."""
+        if self.proc is None:
+            return
+        t0 = time.time()
+        while not self.rows and time.time() - t0 < timeout_s and self.proc.poll() is None:
+            time.sleep(0.02)
+        self.skip = len(self.rows)
 
     def stop(self):
         if self.proc is None:
@@ -70,7 +82,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[self.skip:]:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
                 for n, v in zip(names, r[3:7]):
@@ -275,6 +287,9 @@ def main():
     sampler = ClockSampler(local_rank)      # runs through warm-up, the timed region and the end-to-end region (all under load)
     if rank == 0:
         sampler.start()
+        sampler.wait_until_running()
+    if world > 1:
+        dist.barrier()
     for _ in range(args.warmup):
         step(d)
     B.check_dev_status()
@@ -325,6 +340,12 @@ def main():
         e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
                "ms_per_step": e2e_ms, "inputs": "all operands (queries, keys, weights, Q, KV pool, page table) uploaded every step"}
 
+    # a short run can end between two samples: keep the same load on until one sample has been taken under it
+    if rank == 0 and sampler.proc is not None:
+        t_wait = time.time()
+        while len(sampler.rows) - sampler.skip < 2 and time.time() - t_wait < 2.0:
+            step(d)
+            torch.cuda.synchronize()
     # ---- side measurement (not part of `value`): indexer + top-k as one call that never stores the score matrix
     fused = None
     if not args.no_fused:

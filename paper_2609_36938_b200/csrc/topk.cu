@@ -16,12 +16,14 @@
 namespace janus {
 
 constexpr int TK_CAP = 8192;        // 73 KB of shared memory per CTA keeps three CTAs on an SM
-using TopkShared = TopkSharedT<TK_CAP>;
+constexpr int TK_CAP_SMALL = 5632;  // 54 KB: four CTAs on an SM (all 2048 threads), for rows whose candidate list is sure to fit
 
+template <int CAP>
 __global__ void __launch_bounds__(TK_THREADS)
 topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int k,
                  int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    using TopkShared = TopkSharedT<CAP>;
     TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
     const int t = blockIdx.x;
     int64_t prefix64 = causal ? min(n_keys, q_pos0 + t + 1) : n_keys;
@@ -43,9 +45,24 @@ extern "C" int janus_topk(const float* scores, int64_t scores_ld, int M, int64_t
     if (M == 0) return JANUS_OK;
     if (!idx) return JANUS_ERR_INVALID_ARG;
     if (n_keys > 0 && (!scores || !aligned16(scores) || (scores_ld & 3) != 0)) return JANUS_ERR_INVALID_ARG;
-    const size_t smem = sizeof(TopkShared);
-    JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    topk_rows_kernel<<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+    // The candidate list of a row holds what passes the sampled threshold: about n * r / 4096 elements for the sample rank
+    // r = e + 4 sqrt(e) + 8, e = 4096 k / n, give or take n sqrt(r) / 4096.  When that plus five deviations fits the small
+    // buffer for the longest row, four CTAs share an SM instead of three.
+    const double n_max = static_cast<double>(causal ? (n_keys < q_pos0 + M ? n_keys : q_pos0 + M) : n_keys);
+    bool small = false;
+    if (n_max > TK_CAP) {
+        const double e = 4096.0 * k / n_max, r = e + 4.0 * sqrt(e) + 8.0;
+        small = n_max * (r + 5.0 * sqrt(r)) / 4096.0 <= TK_CAP_SMALL && k <= TK_CAP_SMALL / 2;
+    }
+    if (small) {
+        const size_t smem = sizeof(TopkSharedT<TK_CAP_SMALL>);
+        JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel<TK_CAP_SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        topk_rows_kernel<TK_CAP_SMALL><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+    } else {
+        const size_t smem = sizeof(TopkSharedT<TK_CAP>);
+        JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        topk_rows_kernel<TK_CAP><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+    }
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
