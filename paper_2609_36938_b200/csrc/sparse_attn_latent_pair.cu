@@ -11,27 +11,35 @@
 //   CTA 1 owns row bytes [512,1152) = dims [256,576):  value half 1, and the last 320 dims of the contraction.
 //
 // Each CTA gathers only its own bytes of every selected row, computes a partial logit tile S_c = Q_c . K_c^T
-// (128 heads x 64 keys, fp32 in TMEM), and the two partial tiles are exchanged through distributed shared memory:
-// every softmax thread (thread = head) sends its 64 partial logits into the peer's exchange buffer with asynchronous
-// remote stores that are counted on the peer's mbarrier as they land, waits for the peer's values and adds them.  Both CTAs then run the same fp32 online softmax on
-// identical sums, write P (bf16) back to TMEM over the logits, and accumulate O_c += P . V_c with V_c read MN-major
-// from the gathered rows (the value half of CTA c is the first 256 dims of the bytes it owns).
+// (128 heads x 64 keys, fp32 in tensor memory), and the two partial tiles are exchanged through distributed shared
+// memory: the exchange warps send the 64 partial logits of every head into the peer's exchange buffer with asynchronous
+// remote stores that are counted on the peer's mbarrier as they land.  The partial logits travel as fp16 (11 significant
+// bits; P itself is bf16): the link between the two SMs is the slowest step of the tile loop, and half the bytes also
+// make room for a fourth ring buffer.  Each CTA adds the peer's values to its own fp32 partial logits, runs the fp32
+// online softmax, writes P (bf16) to its own place in tensor memory and accumulates O_c += P . V_c with V_c read
+// MN-major from the gathered rows (the value half of CTA c is the first 256 dims of the bytes it owns).
 //
-// Per CTA: queries live in tensor memory as the A operand (4 atoms of 64 dims = 128 columns; the fifth atom of
-// CTA 1, the 64 rope dims, sits in shared memory); tensor memory = O 256 | two logit buffers of 64 | Q 128 columns.
-// Keys move in half-tiles of 32 rows through a ring of three 64-key tiles.  Warp roles (15 warps):
-//   warp 0       issues the MMAs: S for tile i+1 (16 or 20 MMAs 128x64x16) before O += P.V of tile i (4 MMAs 128x256x16);
-//   warps 1-6    gather: each owns one ring slot, resolves its 32 rows through the page table (one half-tile ahead)
-//                and copies this CTA's bytes with 16-byte cp.async into the 128-byte-swizzled K-major layout;
-//   warps 7-10   exchange: as soon as a partial logit tile is complete they send it to the peer, so the transfer of
-//                tile i+1 overlaps the softmax of tile i; after a token's last tile they load the next token's queries;
-//   warps 11-14  softmax (thread = head): add the peer's partial logits, fp32 online softmax, write P (bf16) over the logits.
+// Per CTA: tensor memory = O 256 | two logit buffers of 64 | P 32 | queries 96 columns (three atoms of 64 dims as the A
+// operand; the fourth atom, and the 64 rope dims on CTA 1, sit in shared memory).  Keys move in half-tiles of 32 rows
+// through a ring of four 64-key tiles.  Warp roles (12 warps, 168 registers per thread available):
+//   warp 0       issues the MMAs in the order their inputs become ready: a logit tile (12 MMAs 128x64x16 from tensor
+//                memory + 4 or 8 from shared memory) needs its rows and a logit buffer that every reader has in registers,
+//                so it runs about two tiles ahead of the softmax; O += P.V (4 MMAs 128x256x16) needs P;
+//   warps 1-3    gather: warp g owns the ring slots s with s % 3 == g, resolves its 32 rows through the page table (one
+//                half-tile ahead) and copies this CTA's bytes with 16-byte cp.async into the 128-byte-swizzled K-major
+//                layout, 8 rows x 64 bytes per instruction;
+//   warps 4-7    exchange: as soon as a partial logit tile is complete they take it into registers, free the logit
+//                buffer and send it to the peer; after a token's last tile they load the next token's queries (prefetched
+//                into L2 one token earlier);
+//   warps 8-11   softmax (thread = head): add the peer's partial logits, fp32 online softmax, write P.
 // The kernel is persistent: one cluster per SM pair loops over tokens, and the ring, the logit buffers and all barrier
 // phases run on across tokens, so a token's prologue (queries into tensor memory, first gathers) hides behind the previous
 // token's last tiles and output.
-// The running max only moves when a tile exceeds it by more than 2^8, so O is rescaled (in TMEM) a handful of times
-// per row.  Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT, and both CTAs of the cluster
-// still meet at the final cluster barrier.
+// The running max only moves when a tile exceeds it by more than 2^8, so O is rescaled (in tensor memory) a handful of
+// times per row.  Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT, and both CTAs of the
+// cluster still meet at the final cluster barrier.
+#include <cuda_fp16.h>
+
 #include "janus_common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -45,28 +53,34 @@ constexpr int LP_DV = 512;
 constexpr int LP_DVH = 256;
 constexpr int LP_HALF = 32;                 // rows per half-tile (gather / ring-slot granularity)
 constexpr int LP_TILE = 2 * LP_HALF;        // keys per MMA tile
-constexpr int LP_BUFS = 3;                  // 64-key tile buffers
+constexpr int LP_BUFS = 4;                  // 64-key tile buffers
 constexpr int LP_SLOTS = 2 * LP_BUFS;       // ring slots (half-tiles)
-constexpr int LP_GATHER_WARPS = 3;          // warp g owns ring slots g and g + 3 (must divide LP_SLOTS); 12 warps in all leave
+constexpr int LP_GATHER_WARPS = 3;          // warp g owns the ring slots s with s % 3 == g; 12 warps in all leave
                                             // 168 registers per thread, which the softmax needs to stay out of local memory
 constexpr int LP_ATOMS_MAX = 5;             // 64-dim atoms owned by a CTA: 4 (CTA 0) or 5 (CTA 1)
 constexpr int LP_K_ATOM_BYTES = LP_TILE * 128;                   // 8 KB
 constexpr int LP_TILE_BYTES = LP_ATOMS_MAX * LP_K_ATOM_BYTES;    // 40 KB
-constexpr int LP_XBUF_BYTES = LP_TILE * LP_HEADS * 4;            // 32 KB: partial logits from the peer, [key/4][head][4] fp32
+constexpr int LP_XBUF_BYTES = LP_TILE * LP_HEADS * 2;            // 16 KB: partial logits from the peer, [key/8][head][8] fp16
 constexpr int LP_Q_ATOM_BYTES = LP_HEADS * 128;                  // 16 KB
 constexpr int LP_XCHG_WARP0 = 1 + LP_GATHER_WARPS;               // first exchange warp
 constexpr int LP_SMAX_WARP0 = LP_XCHG_WARP0 + 4;                 // first softmax warp
 constexpr int LP_THREADS = 32 * (LP_SMAX_WARP0 + 4);             // 12 warps
-constexpr uint32_t LP_COL_O = 0, LP_COL_S = 256, LP_COL_Q = 384;
+constexpr int LP_Q_TMEM_ATOMS = 3;                               // query atoms kept in tensor memory; the others sit in shared memory
+constexpr int LP_QS_BYTES = 2 * LP_Q_ATOM_BYTES;                 // 32 KB: owned query atom 3 (and 4 on CTA 1)
+constexpr uint32_t LP_COL_O = 0, LP_COL_S = 256, LP_COL_P = 384, LP_COL_Q = 416;   // O 256 | 2 x 64 logits | P 32 | 3 x 32 query
 
 struct LpShared {
     uint64_t q_full, qt_full;
     uint64_t k_full[LP_BUFS], k_empty[LP_BUFS];   // per tile buffer: rows landed (2 half-tiles) / P.V of the tile done
-    uint64_t s_full[2], p_full[2];
+    uint64_t s_full[2];                           // logits of the tile using logit buffer b are complete
+    uint64_t s_free[2];                           // every reader (4 softmax + 4 exchange warps) has logit buffer b in registers
+    uint64_t p_full;                              // P of the tile is in tensor memory
     uint64_t x_full[2];                           // the peer's partial logits of the tile using logit buffer b have arrived
     uint64_t x_empty[2];                          // the PEER has read this CTA's previous partial logits out of its exchange buffer b
-    uint64_t x_sent[2];                           // this CTA's exchange warps have read logit buffer b (P may overwrite it)
     uint32_t vmask[LP_SLOTS];
+#ifdef JANUS_ATTN_PROFILE
+    long long prof_ts[2], prof_ts2[2];            // when the exchange warps saw the logits complete / had sent them
+#endif
     uint32_t tmem_base;
     uint32_t start_abort[2];
 };
@@ -111,6 +125,10 @@ __device__ __forceinline__ float lp_exp2(float x) {   // ex2.approx: 2 ulp, exp2
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ uint32_t lp_pack_f16x2(float lo, float hi) {   // saturating: a logit beyond the fp16 range stays finite
+    const __half2 v = __floats2half2_rn(fminf(fmaxf(lo, -65504.f), 65504.f), fminf(fmaxf(hi, -65504.f), 65504.f));
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ uint32_t lp_pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -120,9 +138,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(LP_THREADS, 1)
 sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const LpParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* k_smem = smem;                                              // 3 tiles x 5 atoms x [64 keys x 128 B]
-    float* xbuf = reinterpret_cast<float*>(smem + LP_BUFS * LP_TILE_BYTES);    // 2 x [64 keys][128 heads]
-    unsigned char* q4_smem = smem + LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES;   // CTA 1: query dims [512,576)
-    LpShared* sh = reinterpret_cast<LpShared*>(q4_smem + LP_Q_ATOM_BYTES);
+    unsigned char* xbuf = smem + LP_BUFS * LP_TILE_BYTES;                      // 2 x [64 keys / 8][128 heads][8 keys] fp16
+    unsigned char* q_smem = smem + LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES;    // owned query atom 3 (and 4 on CTA 1), each [128 heads x 128 B]
+    LpShared* sh = reinterpret_cast<LpShared*>(q_smem + LP_QS_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t c = cluster_ctarank();          // 0 or 1: which bytes of the rows this CTA owns
@@ -142,11 +160,11 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         for (int s = 0; s < LP_BUFS; ++s) { mbar_init(smem_u32(&sh->k_full[s]), 2); mbar_init(smem_u32(&sh->k_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh->s_full[b]), 1);
-            mbar_init(smem_u32(&sh->p_full[b]), 4);
+            mbar_init(smem_u32(&sh->s_free[b]), 8);
             mbar_init(smem_u32(&sh->x_full[b]), 1);
             mbar_init(smem_u32(&sh->x_empty[b]), 4);
-            mbar_init(smem_u32(&sh->x_sent[b]), 4);
         }
+        mbar_init(smem_u32(&sh->p_full), 4);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         // start-up agreement: if this CTA should not start (misaligned shared memory, or an earlier CTA of the launch gave
@@ -171,85 +189,90 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
     if (start_abort) {
         // nothing to do
     } else if (warp == 0) {
-        // ================================================================== MMA issue (whole warp runs the loop, lane 0 issues)
-        const bool leader = lane == 0;
+        // ================================================================== MMA issue
+        // Lane 0 runs the whole role.  Logit tiles and P.V products are issued in whatever order their inputs become
+        // ready (P.V first when both are).  P has a place of its own in tensor memory, so a logit tile only needs its rows
+        // and a logit buffer whose previous contents every reader holds in registers: it is issued while the softmax of
+        // two tiles earlier is still running, and the softmax does not wait for the tensor pipe to turn around.
         const uint32_t qf = smem_u32(&sh->q_full);
-        auto fetch_q4 = [&](int it) {      // rope dims [512,576) of all heads of this cluster's token `it` (CTA 1 only)
-            if (!leader) return;
-            if (c == 1u) {
-                mbar_expect_tx(qf, LP_Q_ATOM_BYTES);
-                tma_load_2d(smem_u32(q4_smem), &tmap_q, 512, (cid + it * n_clusters) * LP_HEADS, qf);
-            } else {
-                mbar_arrive(qf);
-            }
+        auto fetch_q = [&](int it) {       // owned query atom 3 (and 4 on CTA 1) of all heads of this cluster's token `it`
+            const int y = (cid + it * n_clusters) * LP_HEADS;
+            mbar_expect_tx(qf, static_cast<uint32_t>((n_atoms - LP_Q_TMEM_ATOMS) * LP_Q_ATOM_BYTES));
+            tma_load_2d(smem_u32(q_smem), &tmap_q, 256 * static_cast<int>(c) + 64 * LP_Q_TMEM_ATOMS, y, qf);
+            if (c == 1u) tma_load_2d(smem_u32(q_smem + LP_Q_ATOM_BYTES), &tmap_q, 512, y, qf);
         };
-        if (n_my > 0) fetch_q4(0);
-        constexpr uint32_t idesc_qk = umma_idesc_major(1u, LP_HEADS, LP_TILE, 0u, 0u);
-        constexpr uint32_t idesc_pv = umma_idesc_major(1u, LP_HEADS, LP_DVH, 0u, 1u);
-        LP_PROF_DECL(w_kfull); LP_PROF_DECL(w_pfull); LP_PROF_DECL(w_q);
-        const long long prof_t0 = LP_PROF_NOW();
-        const uint32_t q4_lo = umma_desc_lo(smem_u32(q4_smem), 16);
-        const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem), 16);
-        const uint32_t v_lo = umma_desc_lo(smem_u32(k_smem), LP_K_ATOM_BYTES);     // value half = first four owned atoms
-        auto issue_pv = [&](int j, bool first) {   // O += P_j . V_j (j counts tiles globally; `first`: the token's first tile)
-            const int b = j & 1, buf = j % LP_BUFS;
-            const uint32_t vb = v_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
-            const uint32_t pa = tmem_base + LP_COL_S + b * LP_TILE;
-            if (leader) {
-#pragma unroll
-                for (int ks = 0; ks < LP_TILE / 16; ++ks)
-                    umma_bf16_ts_lohi(tmem_base + LP_COL_O, pa + ks * 8, vb + ks * (2048 >> 4), idesc_pv, (!first || ks > 0) ? 1u : 0u);
-                umma_commit(smem_u32(&sh->k_empty[buf]));   // tile buffer free again, and "P.V of tile j done" for the softmax warps
-            }
-        };
-        bool ok = true;
-        int gi = 0;                                  // tiles issued so far, over all tokens
-        for (int it = 0; it < n_my && ok; ++it) {
-            ok = LP_PROF_WAIT(w_q, mbar_wait(qf, static_cast<uint32_t>(it) & 1u) && mbar_wait(smem_u32(&sh->qt_full), static_cast<uint32_t>(it) & 1u));
-            if (!ok) break;
-            tc_fence_after();
-            for (int i = 0; i < n_tiles; ++i, ++gi) {
-                const int b = gi & 1, buf = gi % LP_BUFS;
-                ok = LP_PROF_WAIT(w_kfull, mbar_wait(smem_u32(&sh->k_full[buf]), static_cast<uint32_t>(gi / LP_BUFS) & 1u));
+        if (lane == 0) {
+            if (n_my > 0) fetch_q(0);
+            constexpr uint32_t idesc_qk = umma_idesc_major(1u, LP_HEADS, LP_TILE, 0u, 0u);
+            constexpr uint32_t idesc_pv = umma_idesc_major(1u, LP_HEADS, LP_DVH, 0u, 1u);
+            LP_PROF_DECL(w_kfull); LP_PROF_DECL(w_pfull); LP_PROF_DECL(w_q);
+            const long long prof_t0 = LP_PROF_NOW();
+            const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem), 16);
+            const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem), 16);
+            const uint32_t v_lo = umma_desc_lo(smem_u32(k_smem), LP_K_ATOM_BYTES);     // value half = first four owned atoms
+            bool ok = true;
+            int s_next = 0, pv_next = 0;                 // next logit tile / next P.V to issue, counted over all tokens
+            for (int it = 0; it < n_my && ok; ++it) {
+                ok = LP_PROF_WAIT(w_q, mbar_wait(qf, static_cast<uint32_t>(it) & 1u) && mbar_wait(smem_u32(&sh->qt_full), static_cast<uint32_t>(it) & 1u));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_s = tmem_base + LP_COL_S + b * LP_TILE;
-                const uint32_t kb = k_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
-                if (leader) {
+                const int tok_begin = it * n_tiles, tok_end = tok_begin + n_tiles;
+                uint32_t idle = 0;
+                while (pv_next < tok_end) {
+                    if (pv_next < s_next && mbar_test_wait(smem_u32(&sh->p_full), static_cast<uint32_t>(pv_next) & 1u)) {
+                        // O += P_j . V_j
+                        tc_fence_after();
+                        const int j = pv_next, buf = j % LP_BUFS;
+                        const uint32_t vb = v_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) {
+                        for (int ks = 0; ks < LP_TILE / 16; ++ks)
+                            umma_bf16_ts_lohi(tmem_base + LP_COL_O, tmem_base + LP_COL_P + ks * 8, vb + ks * (2048 >> 4), idesc_pv,
+                                              (j > tok_begin || ks > 0) ? 1u : 0u);
+                        umma_commit(smem_u32(&sh->k_empty[buf]));   // tile buffer and P free again; "P.V of tile j done" for the softmax warps
+                        ++pv_next;
+                        idle = 0;
+                    } else if (s_next < tok_end && mbar_test_wait(smem_u32(&sh->k_full[s_next % LP_BUFS]), static_cast<uint32_t>(s_next / LP_BUFS) & 1u) &&
+                               (s_next < 2 || mbar_test_wait(smem_u32(&sh->s_free[s_next & 1]), static_cast<uint32_t>((s_next - 2) >> 1) & 1u))) {
+                        // S_j = Q . K_j^T into logit buffer j & 1
+                        tc_fence_after();
+                        const int b = s_next & 1, buf = s_next % LP_BUFS;
+                        const uint32_t d_s = tmem_base + LP_COL_S + b * LP_TILE;
+                        const uint32_t kb = k_lo + static_cast<uint32_t>(buf * (LP_TILE_BYTES >> 4));
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            umma_bf16_ts_lohi(d_s, tmem_base + LP_COL_Q + a * 32 + ks * 8, kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk,
-                                              (a > 0 || ks > 0) ? 1u : 0u);
+                        for (int a = 0; a < LP_Q_TMEM_ATOMS; ++a) {
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16_ts_lohi(d_s, tmem_base + LP_COL_Q + a * 32 + ks * 8, kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk,
+                                                  (a > 0 || ks > 0) ? 1u : 0u);
+                        }
+#pragma unroll
+                        for (int a = LP_Q_TMEM_ATOMS; a < LP_ATOMS_MAX; ++a) {
+                            if (a < n_atoms) {
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks)
+                                    umma_bf16_ss_lohi(d_s, q_lo + (a - LP_Q_TMEM_ATOMS) * (LP_Q_ATOM_BYTES >> 4) + ks * 2,
+                                                      kb + a * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk, 1u);
+                            }
+                        }
+                        umma_commit(smem_u32(&sh->s_full[b]));
+                        ++s_next;
+                        idle = 0;
+                    } else if (++idle > (1u << 24)) {     // nothing became ready for about a second: give up
+                        ok = false;
+                        break;
                     }
-                    if (c == 1u) {
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            umma_bf16_ss_lohi(d_s, q4_lo + ks * 2, kb + 4 * (LP_K_ATOM_BYTES >> 4) + ks * 2, idesc_qk, 1u);
-                    }
-                    umma_commit(smem_u32(&sh->s_full[b]));
                 }
-                if (i >= 1) {
-                    ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(gi - 1) & 1]), static_cast<uint32_t>((gi - 1) >> 1) & 1u));
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(gi - 1, i == 1);
-                }
+                if (!ok) break;
+                // every P of the token exists, so every logit MMA of the token has completed: its queries may be replaced;
+                // the output of the token is read out of O before the softmax warps produce the next token's first P
+                if (it + 1 < n_my) fetch_q(it + 1);
             }
-            if (!ok) break;
-            // the token's last P: once it exists, every logit MMA of the token has completed, so the queries may be replaced;
-            // the output of the token has been read out of O before the softmax warps produce the next token's first P
-            ok = LP_PROF_WAIT(w_pfull, mbar_wait(smem_u32(&sh->p_full[(gi - 1) & 1]), static_cast<uint32_t>((gi - 1) >> 1) & 1u));
-            if (!ok) break;
-            tc_fence_after();
-            issue_pv(gi - 1, n_tiles == 1);
-            if (it + 1 < n_my) fetch_q4(it + 1);
+            if (!ok) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+            LP_PROF_PUT(0, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(1, w_kfull); LP_PROF_PUT(2, w_pfull); LP_PROF_PUT(9, w_q);
         }
-        if (!ok && leader) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
-        if (leader) { LP_PROF_PUT(0, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(1, w_kfull); LP_PROF_PUT(2, w_pfull); LP_PROF_PUT(9, w_q); }
+        __syncwarp();
     } else if (warp <= LP_GATHER_WARPS) {
-        // ================================================================== gather: warp g owns ring slot g (half-tiles g, g+6, ...)
+        // ================================================================== gather: warp g owns the ring slots s with s % 3 == g
         // A warp copies whole half-tiles (32 rows, this CTA's bytes of each), so address resolution is done once per
         // half-tile and no two warps ever synchronise.  Because every use of a slot is made by the same warp, the slot's
         // barrier is at most one phase ahead of it, which the parity wait relies on.
@@ -283,11 +306,16 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             return ptr;
         };
         // rows are resolved one half-tile ahead and indices fetched two ahead, so neither load is waited for in the loop
+        auto next_owned = [&](int gh) -> int {                 // the next half-tile after gh whose ring slot this warp owns
+            do { ++gh; } while ((gh & (LP_SLOTS - 1)) % LP_GATHER_WARPS != g);
+            return gh;
+        };
         bool valid_cur, valid_nxt = false;
         const unsigned char* row_ptr = resolve(load_raw(g), valid_cur);
         const unsigned char* row_nxt = row_ptr;
-        int raw_nxt = load_raw(g + LP_GATHER_WARPS);
-        for (int hi = g; hi < total_half; hi += LP_GATHER_WARPS) {
+        int hi_nxt = next_owned(g);
+        int raw_nxt = load_raw(hi_nxt);
+        for (int hi = g; hi < total_half; hi = hi_nxt, hi_nxt = next_owned(hi_nxt)) {
             const int buf = (hi >> 1) % LP_BUFS, hf = hi & 1;
             const bool s_ok = valid_cur;
             const uint32_t valid_mask = __ballot_sync(0xffffffffu, s_ok);
@@ -317,7 +345,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             }
             cp_async_commit();
             row_nxt = resolve(raw_nxt, valid_nxt);                 // page-table load overlaps the copies in flight
-            raw_nxt = load_raw(hi + 2 * LP_GATHER_WARPS);
+            raw_nxt = load_raw(next_owned(hi_nxt));
             LP_PROF_WAIT(w_group, (cp_async_wait<0>(), true));
             fence_proxy_async();              // publish the landed rows to the MMA (async) proxy
             __syncwarp();
@@ -329,7 +357,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         if (g == 0 && lane == 0) { LP_PROF_PUT(3, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(4, w_kempty); LP_PROF_PUT(5, w_group); }
     } else if (warp < LP_SMAX_WARP0) {
         // ================================================================== exchange: partial logits -> the peer's buffer
-        const int quad = warp & 3;                         // warps 7..10 -> TMEM lane quadrants 3,0,1,2
+        const int quad = warp & 3;                         // warps 4..7 -> TMEM lane quadrants 0..3
         const int h = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const uint32_t peer_xbuf = mapa_shared(smem_u32(xbuf), peer);
@@ -338,7 +366,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         auto load_q = [&](int it) {
             const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<int64_t>(cid + it * n_clusters) * LP_HEADS + h) * LP_DQK + 256 * c);
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
+            for (int a = 0; a < LP_Q_TMEM_ATOMS; ++a) {
                 uint32_t r[32];
 #pragma unroll
                 for (int v = 0; v < 8; ++v) {
@@ -365,30 +393,49 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         for (int i = 0; i < n_tiles; ++i, ++gi) {
             const int b = gi & 1;
             const uint32_t ph = static_cast<uint32_t>(gi >> 1) & 1u;
-            // the logits are complete, and the peer has read what this CTA sent two tiles ago into the same buffer
-            ok = mbar_wait(smem_u32(&sh->s_full[b]), ph) && mbar_wait(smem_u32(&sh->x_empty[b]), ph ^ 1u);
+            ok = mbar_wait(smem_u32(&sh->s_full[b]), ph);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+#ifdef JANUS_ATTN_PROFILE
+            if (warp == LP_XCHG_WARP0 && lane == 0) sh->prof_ts[b] = clock64();
+#endif
             const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
-            // [key/4][head][4 keys] fp32: a warp stores 512 contiguous bytes per instruction; every 16 bytes are counted
-            // on the peer's barrier when they land, so nothing here waits for the transfer
+            uint32_t r0[32], r1[32];
+            tmem_ld32_issue(s_addr, r0);
+            tmem_ld32_issue(s_addr + 32, r1);
+            tmem_ld_wait(r0);
+            tmem_ld_wait(r1);
+            // the partial logits are in registers: the logit buffer may take the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
+            // the peer must have read what this CTA sent two tiles ago into the same exchange buffer
+            ok = mbar_wait(smem_u32(&sh->x_empty[b]), ph ^ 1u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            // The partial logits travel as fp16 (11 significant bits: the same order of rounding as P, which is bf16), which
+            // halves the traffic between the two SMs, the slowest link of the tile loop.  [key/8][head][8 keys]: a warp
+            // stores 512 contiguous bytes per instruction; every 16 bytes are counted on the peer's barrier when they land.
             const uint32_t dst = peer_xbuf + static_cast<uint32_t>(b * LP_XBUF_BYTES + h * 16);
             const uint32_t bar = peer_xfull + static_cast<uint32_t>(b * 8);
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t r[32];
-                tmem_ld32_wait(s_addr + hf * 32, r);
-                if (hf == 1) {   // both halves are in registers: the softmax warps may overwrite the logits with P
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh->x_sent[b]));
-                }
+            for (int j8 = 0; j8 < 4; ++j8)
+                st_async_cluster_f32x4(dst + static_cast<uint32_t>(j8 * LP_HEADS * 16),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r0[8 * j8]), __uint_as_float(r0[8 * j8 + 1]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r0[8 * j8 + 2]), __uint_as_float(r0[8 * j8 + 3]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r0[8 * j8 + 4]), __uint_as_float(r0[8 * j8 + 5]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r0[8 * j8 + 6]), __uint_as_float(r0[8 * j8 + 7]))), bar);
 #pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4)
-                    st_async_cluster_f32x4(dst + static_cast<uint32_t>((hf * 8 + j4) * LP_HEADS * 16), __uint_as_float(r[4 * j4]),
-                                           __uint_as_float(r[4 * j4 + 1]), __uint_as_float(r[4 * j4 + 2]), __uint_as_float(r[4 * j4 + 3]), bar);
-            }
+            for (int j8 = 0; j8 < 4; ++j8)
+                st_async_cluster_f32x4(dst + static_cast<uint32_t>((4 + j8) * LP_HEADS * 16),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8]), __uint_as_float(r1[8 * j8 + 1]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 2]), __uint_as_float(r1[8 * j8 + 3]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 4]), __uint_as_float(r1[8 * j8 + 5]))),
+                                       __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 6]), __uint_as_float(r1[8 * j8 + 7]))), bar);
+#ifdef JANUS_ATTN_PROFILE
+            if (warp == LP_XCHG_WARP0 && lane == 0) sh->prof_ts2[b] = clock64();
+#endif
         }
             // the token's last logit tile is complete, so nothing reads its queries any more: bring in the next token's
             if (ok && it + 1 < n_my) load_q(it + 1);
@@ -403,7 +450,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const bool out_al32 = (reinterpret_cast<uint64_t>(p.out) & 31u) == 0u;
         bool ok = true;
         LP_PROF_DECL(w_sfull); LP_PROF_DECL(w_xfull); LP_PROF_DECL(w_send);
-        LP_PROF_DECL(e_wait); LP_PROF_DECL(e_out);
+        LP_PROF_DECL(e_wait); LP_PROF_DECL(e_out); LP_PROF_DECL(w_x01); LP_PROF_DECL(w_s01); LP_PROF_DECL(x_lat); LP_PROF_DECL(x_lat2);
         LP_PROF_DECL(s_ld); LP_PROF_DECL(s_peer); LP_PROF_DECL(s_arr); LP_PROF_DECL(s_exp); LP_PROF_DECL(s_st);
         const long long prof_t0 = LP_PROF_NOW();
         long long seg = prof_t0;
@@ -421,7 +468,11 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (warp == LP_SMAX_WARP0 && lane == 0) mbar_expect_tx(smem_u32(&sh->x_full[b]), LP_XBUF_BYTES);
             // k_full is complete long before s_full; waiting on it as well makes the validity masks written by the gather
             // warps visible to this thread directly rather than through the MMA warp
-            ok = LP_PROF_WAIT(w_sfull, mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s));
+#ifdef JANUS_ATTN_PROFILE
+            { const long long _t0 = clock64(); ok = mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s); const long long _d = clock64() - _t0; w_sfull += _d; if (i < 2) w_s01 += _d; }
+#else
+            ok = mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s);
+#endif
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -435,20 +486,31 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
 #pragma unroll
                 for (int j = 0; j < 16; ++j) x[hf * 16 + j] = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
             }
+            // the logits are in registers: the logit buffer may take the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
             LP_PROF_SEG(s_ld, seg);
             // the peer's partial logits of the same tile (bytes counted as they land: visible once the phase completes)
-            ok = LP_PROF_WAIT(w_xfull, mbar_wait(smem_u32(&sh->x_full[b]), ph_s));
+#ifdef JANUS_ATTN_PROFILE
+            { const long long _t0 = clock64(); ok = mbar_wait(smem_u32(&sh->x_full[b]), ph_s); const long long _n = clock64(); const long long _d = _n - _t0; w_xfull += _d; if (i < 2) w_x01 += _d;
+              if (_d > 100) { x_lat += _n - *reinterpret_cast<volatile long long*>(&sh->prof_ts[b]); x_lat2 += _n - *reinterpret_cast<volatile long long*>(&sh->prof_ts2[b]); } }
+#else
+            ok = mbar_wait(smem_u32(&sh->x_full[b]), ph_s);
+#endif
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             float tile_max = neg_inf;
             seg = LP_PROF_NOW();
             {
-                const float4* xin = reinterpret_cast<const float4*>(xbuf + b * (LP_XBUF_BYTES / 4)) + h;
+                const uint4* xin = reinterpret_cast<const uint4*>(xbuf + b * LP_XBUF_BYTES) + h;
 #pragma unroll
-                for (int j4 = 0; j4 < LP_TILE / 4; ++j4) {
-                    const float4 pv = xin[j4 * LP_HEADS];
-                    x[2 * j4] = fadd2(x[2 * j4], make_float2(pv.x, pv.y));
-                    x[2 * j4 + 1] = fadd2(x[2 * j4 + 1], make_float2(pv.z, pv.w));
+                for (int j8 = 0; j8 < LP_TILE / 8; ++j8) {
+                    const uint4 pv = xin[j8 * LP_HEADS];
+                    x[4 * j8 + 0] = fadd2(x[4 * j8 + 0], __half22float2(*reinterpret_cast<const __half2*>(&pv.x)));
+                    x[4 * j8 + 1] = fadd2(x[4 * j8 + 1], __half22float2(*reinterpret_cast<const __half2*>(&pv.y)));
+                    x[4 * j8 + 2] = fadd2(x[4 * j8 + 2], __half22float2(*reinterpret_cast<const __half2*>(&pv.z)));
+                    x[4 * j8 + 3] = fadd2(x[4 * j8 + 3], __half22float2(*reinterpret_cast<const __half2*>(&pv.w)));
                 }
                 const uint32_t vm0 = sh->vmask[2 * buf], vm1 = sh->vmask[2 * buf + 1];
                 if ((vm0 & vm1) != 0xffffffffu) {
@@ -515,14 +577,17 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             const float tile_sum = t4.x + t4.y;
             l_sum += tile_sum;
             LP_PROF_SEG(s_exp, seg);
-            // P overwrites the first 32 columns of the logits: the exchange warps must have read them
-            ok = mbar_wait(smem_u32(&sh->x_sent[b]), ph_s);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tmem_st32_wait(s_addr, pk);
+            // P has one buffer: the previous tile's P.V must have completed
+            if (gi > 0) {
+                ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            tmem_st32_wait(lane_addr + LP_COL_P, pk);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->p_full[b]));
+            if (lane == 0) mbar_arrive(smem_u32(&sh->p_full));
             LP_PROF_SEG(s_st, seg);
         }
         if (!ok) break;
@@ -566,7 +631,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         }
         if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
 #ifdef JANUS_ATTN_PROFILE
-        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); LP_PROF_PUT(16, e_wait); LP_PROF_PUT(17, e_out); }
+        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); LP_PROF_PUT(16, e_wait); LP_PROF_PUT(17, e_out); LP_PROF_PUT(18, w_x01); LP_PROF_PUT(19, w_s01); LP_PROF_PUT(20, x_lat); LP_PROF_PUT(21, x_lat2); }
 #endif
     }
     tc_fence_before();
@@ -612,7 +677,8 @@ int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t
     CUtensorMap tq;
     if (!make_tmap_2d_sw128(&tq, q, 2, static_cast<uint64_t>(M) * LP_HEADS, LP_DQK, static_cast<uint64_t>(LP_DQK) * 2, LP_HEADS, 64))
         return JANUS_ERR_CUDA;
-    const size_t smem = LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES + LP_Q_ATOM_BYTES + sizeof(LpShared) + 16;
+    const size_t smem = LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES + LP_QS_BYTES + sizeof(LpShared) + 16;
+    static_assert(LP_BUFS * LP_TILE_BYTES + 2 * LP_XBUF_BYTES + LP_QS_BYTES + sizeof(LpShared) + 16 <= 227 * 1024, "shared memory");
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(sparse_attn_latent_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     // persistent launch: as many 2-CTA clusters as the device keeps resident at once (one CTA per SM), each looping over tokens
     static int resident_clusters[64] = {};
