@@ -234,6 +234,61 @@ int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk,
                               void* out, float* lse,
                               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/*
+ * Decode step over a batch of sessions (Sec. 2.2, "Decode phase"): one new token per session, processed like an append
+ * prefill with a single appended token.  Session b has its own history, so the per-session arrays are concatenated and
+ * addressed through offsets held in device memory:
+ *
+ *   key_offsets    [B + 1] int64: session b's indexer keys (cached history plus the new token's own key) are rows
+ *                  key_offsets[b] .. key_offsets[b+1] of k_idx; every offset is a multiple of 4 (pad between sessions),
+ *                  so that score rows stay 16-byte aligned.  k_scale / col_bias / scores use the same row numbering.
+ *   table_offsets  [B + 1] int64: session b's page table is page_tables[table_offsets[b] .. table_offsets[b+1]);
+ *                  physical page ids are global (one KV pool for all sessions).
+ *
+ * janus_indexer_scores_batch   scores[key_offsets[b] + s] = indexer score of session b's query against its key s
+ *                              (no causal mask: the new token sees all of its session's keys).  q_idx [B, H_I, D_I]
+ *                              contiguous, w [B, H_I], q_scale [B, H_I] or [H_I]; max_keys = an upper bound of the
+ *                              longest session (host value, sizes the launch); total_keys = rows of k_idx.
+ *                              Tensor-core path only: H_I = 64 and 128- or 256-byte rows, else JANUS_ERR_UNSUPPORTED.
+ * janus_topk_batch             idx[b, 0:k) = top-k of the row_lengths[b] scores starting at scores[row_offsets[b]] (positions inside
+ *                              the session, -1 padded), count / kth as in janus_topk.  row_offsets [B + 1] and row_lengths
+ *                              [B] are int64 device arrays; row_lengths may be NULL (rows then run up to the next offset);
+ *                              offsets are multiples of 4.
+ * janus_page_demand_batch      janus_page_demand over all rows at once: row r marks page_tables[table_offsets[r] + s / page_size]
+ *                              for its selected tokens s < demand_limits[r] (the session's cached history length) into one
+ *                              bitmap over the global pool; lists, runs and the miss set against `predicted_bitmap` (for
+ *                              decode: the pages already resident) as in janus_page_demand.
+ * janus_sparse_attn_decode     janus_sparse_attn_prefill with one query row per session and per-row page tables.
+ */
+int janus_indexer_scores_batch(const void* q_idx, const void* k_idx, int64_t k_stride_tok,
+                               const float* w,
+                               const float* q_scale, int64_t q_scale_stride_tok,
+                               const float* k_scale,
+                               const float* row_bias, const float* col_bias,
+                               int B, int H_I, int D_I,
+                               const int64_t* key_offsets, int64_t total_keys, int64_t max_keys,
+                               int dtype, float* scores, int32_t* dev_status, void* stream);
+int janus_topk_batch(const float* scores, const int64_t* row_offsets, const int64_t* row_lengths, int B, int k,
+                     int32_t* idx, int32_t* count, float* kth, int32_t* dev_status, void* stream);
+int janus_page_demand_batch(const int32_t* idx, int64_t n_rows, int k,
+                            const int64_t* demand_limits, int page_size,
+                            const int32_t* page_tables, const int64_t* table_offsets, int64_t n_phys_pages,
+                            const uint32_t* predicted_bitmap,
+                            uint32_t* bitmap,
+                            int32_t* pages, int32_t* n_pages,
+                            int32_t* runs, int32_t* n_runs,
+                            int32_t* miss_pages, int32_t* n_miss,
+                            int32_t* miss_runs, int32_t* n_miss_runs,
+                            int64_t capacity, int32_t* dev_status, void* stream);
+int janus_sparse_attn_decode(const void* q, int B, int H_q, int d_qk,
+                             const void* k_pool, const void* v_pool,
+                             int64_t page_stride, int64_t tok_stride, int64_t head_stride,
+                             int n_kv_heads, int d_v,
+                             const int32_t* idx, int k, int page_size,
+                             const int32_t* page_tables, const int64_t* table_offsets,
+                             float softmax_scale, void* out, float* lse,
+                             int32_t* dev_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,6 +28,7 @@ EXPORTS = [
     "janus_indexer_topk_workspace_size", "janus_indexer_topk", "janus_indexer_topk_static",
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
+    "janus_indexer_scores_batch", "janus_topk_batch", "janus_page_demand_batch", "janus_sparse_attn_decode",
 ]
 
 
@@ -78,6 +79,16 @@ def load() -> ctypes.CDLL:
     lib.janus_sparse_attn_prefill.restype = c_i
     lib.janus_sparse_attn_prefill.argtypes = [c_p, c_i, c_i, c_i, c_p, c_p, c_i64, c_i64, c_i64, c_i, c_i, c_p, c_i, c_i, c_p, c_i64,
                                               c_f, c_p, c_p, c_p, c_sz, c_p, c_p]
+    lib.janus_indexer_scores_batch.restype = c_i
+    lib.janus_indexer_scores_batch.argtypes = [c_p, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_p, c_i64, c_i64, c_i, c_p, c_p, c_p]
+    lib.janus_topk_batch.restype = c_i
+    lib.janus_topk_batch.argtypes = [c_p, c_p, c_p, c_i, c_i, c_p, c_p, c_p, c_p, c_p]
+    lib.janus_page_demand_batch.restype = c_i
+    lib.janus_page_demand_batch.argtypes = [c_p, c_i64, c_i, c_p, c_i, c_p, c_p, c_i64, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_i64,
+                                            c_p, c_p]
+    lib.janus_sparse_attn_decode.restype = c_i
+    lib.janus_sparse_attn_decode.argtypes = [c_p, c_i, c_i, c_i, c_p, c_p, c_i64, c_i64, c_i64, c_i, c_i, c_p, c_i, c_i, c_p, c_p, c_f, c_p, c_p,
+                                             c_p, c_p]
     _lib = lib
     return lib
 
@@ -280,6 +291,87 @@ def janus_sparse_attn_prefill(q: torch.Tensor, k_pool: torch.Tensor, v_pool: tor
                                        page_table.numel(), float(softmax_scale), _ptr(out), _ptr(lse), None, 0,
                                        _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_sparse_attn_prefill")
+    return out, lse
+
+
+# ---- decode step over a batch of sessions -------------------------------------------------------------------------
+def janus_indexer_scores_batch(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, key_offsets: torch.Tensor, max_keys: int, *,
+                               q_scale: Optional[torch.Tensor] = None, k_scale: Optional[torch.Tensor] = None,
+                               row_bias: Optional[torch.Tensor] = None, col_bias: Optional[torch.Tensor] = None,
+                               scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One query row per session against that session's keys.  q_idx [B,H,D]; k_idx [total_keys, D] (sessions concatenated);
+    key_offsets [B+1] int64 on the device.  Returns scores [total_keys] fp32 in the same row numbering as k_idx."""
+    lib = load()
+    B_, H, D = q_idx.shape
+    total = k_idx.shape[0]
+    dtype = _idx_dtype_code(q_idx)
+    if scores is None:
+        scores = torch.empty((total,), dtype=torch.float32, device=q_idx.device)
+    qs_stride = H if (q_scale is not None and q_scale.dim() == 2) else 0
+    rc = lib.janus_indexer_scores_batch(_ptr(q_idx), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
+                                        _ptr(row_bias), _ptr(col_bias), B_, H, D, _ptr(key_offsets), total, int(max_keys), dtype,
+                                        _ptr(scores), _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_indexer_scores_batch")
+    return scores
+
+
+def janus_topk_batch(scores: torch.Tensor, row_offsets: torch.Tensor, k: int, *, row_lengths: Optional[torch.Tensor] = None,
+                     want_count: bool = True, want_kth: bool = True):
+    """Top-k of every ragged row scores[row_offsets[b] : row_offsets[b] + row_lengths[b]] (up to the next offset when
+    row_lengths is None).  Returns (idx [B,k], count | None, kth | None)."""
+    lib = load()
+    B_ = row_offsets.numel() - 1
+    idx = torch.empty((B_, k), dtype=torch.int32, device=scores.device)
+    count = torch.empty((B_,), dtype=torch.int32, device=scores.device) if want_count else None
+    kth = torch.empty((B_,), dtype=torch.float32, device=scores.device) if want_kth else None
+    rc = lib.janus_topk_batch(_ptr(scores), _ptr(row_offsets), _ptr(row_lengths), B_, int(k), _ptr(idx), _ptr(count), _ptr(kth), _ptr(dev_status_tensor()),
+                              _stream())
+    _check(rc, "janus_topk_batch")
+    return idx, count, kth
+
+
+def janus_page_demand_batch(idx: torch.Tensor, *, demand_limits: torch.Tensor, page_size: int, page_tables: torch.Tensor,
+                            table_offsets: torch.Tensor, n_phys_pages: int, predicted_bitmap: Optional[torch.Tensor] = None,
+                            capacity: Optional[int] = None, want_miss: bool = True):
+    """janus_page_demand over rows that each have their own page table and history length (int64 device tensors)."""
+    lib = load()
+    dev = idx.device
+    n_rows, k = idx.shape
+    cap = int(capacity) if capacity is not None else int(n_phys_pages)
+    n_words = (n_phys_pages + 31) // 32
+    out = {
+        "bitmap": torch.empty((n_words,), dtype=torch.int32, device=dev),
+        "pages": torch.empty((max(cap, 1),), dtype=torch.int32, device=dev),
+        "runs": torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev),
+        "counts": torch.zeros((4,), dtype=torch.int32, device=dev),   # n_pages, n_runs, n_miss, n_miss_runs
+    }
+    cp = out["counts"].data_ptr()
+    miss_args = [None, None, None, None]
+    if want_miss:
+        out["miss_pages"] = torch.empty((max(cap, 1),), dtype=torch.int32, device=dev)
+        out["miss_runs"] = torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev)
+        miss_args = [_ptr(out["miss_pages"]), cp + 8, _ptr(out["miss_runs"]), cp + 12]
+    rc = lib.janus_page_demand_batch(_ptr(idx), n_rows, k, _ptr(demand_limits), int(page_size), _ptr(page_tables), _ptr(table_offsets),
+                                     int(n_phys_pages), _ptr(predicted_bitmap), _ptr(out["bitmap"]), _ptr(out["pages"]), cp, _ptr(out["runs"]),
+                                     cp + 4, *miss_args, cap, _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_page_demand_batch")
+    return out
+
+
+def janus_sparse_attn_decode(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, idx: torch.Tensor, *, page_tables: torch.Tensor,
+                             table_offsets: torch.Tensor, page_size: int, softmax_scale: float, d_v: int, want_lse: bool = True,
+                             out: Optional[torch.Tensor] = None):
+    """janus_sparse_attn_prefill with one query row per session and per-row page tables (table_offsets [B+1] int64)."""
+    lib = load()
+    B_, H_q, d_qk = q.shape
+    n_kv = k_pool.shape[2]
+    if out is None:
+        out = torch.empty((B_, H_q, d_v), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B_, H_q), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = lib.janus_sparse_attn_decode(_ptr(q), B_, H_q, d_qk, _ptr(k_pool), _ptr(v_pool), k_pool.stride(0), k_pool.stride(1), k_pool.stride(2),
+                                      n_kv, int(d_v), _ptr(idx), idx.shape[1], int(page_size), _ptr(page_tables), _ptr(table_offsets),
+                                      float(softmax_scale), _ptr(out), _ptr(lse), _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_sparse_attn_decode")
     return out, lse
 
 

@@ -53,6 +53,9 @@ struct TcCandParams {
     int32_t* cand_cnt;    // [M] candidates appended so far (may exceed cand_cap: only the first cand_cap are stored)
     int2* cand;           // [M, cand_cap] (score bits, key index)
     int cand_cap;
+    // ragged batch mode (decode over many sessions): query row b scores the keys key_offsets[b] .. key_offsets[b+1] of one
+    // concatenated key array, no causal mask, and its scores go to scores[key_offsets[b] + s]
+    const int64_t* key_offsets;
 };
 
 // Candidate mode stages appends in shared memory: each epilogue warp owns, for each of its (at most TC_CAND_TPW) tokens,
@@ -101,7 +104,7 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
     }
 }
 
-template <int H, bool FP8, bool CAND>
+template <int H, bool FP8, bool CAND, bool RAGGED>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p, const TcCandParams cp) {
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -119,10 +122,19 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tpc = nq * TPS;                                   // tokens per CTA
-    const int t0 = blockIdx.y * tpc;
+    int t0 = blockIdx.y * tpc;
+    int64_t key_base = 0, key_count = p.n_keys;                 // this CTA's keys: rows key_base .. key_base + key_count of k_idx
+    int n_tiles = p.n_tiles;
+    if constexpr (RAGGED) {
+        t0 = blockIdx.y;                                        // one query row per grid row; the sub-tile's other rows are not stored
+        key_base = cp.key_offsets[blockIdx.y];
+        key_count = cp.key_offsets[blockIdx.y + 1] - key_base;
+        if (key_count < 0) key_count = 0;
+        n_tiles = static_cast<int>((key_count + TC_KEYS - 1) / TC_KEYS);
+    }
     const int t_hi = min(p.M, t0 + tpc) - 1;                    // last real token of this CTA
     const int tile_begin = blockIdx.x * p.tiles_per_cta;
-    const int tile_end = min(p.n_tiles, tile_begin + p.tiles_per_cta);
+    const int tile_end = min(n_tiles, tile_begin + p.tiles_per_cta);
     // key tiles with at least one visible (token, key) pair come first
     int vis_end = tile_end;
     if (p.causal) {
@@ -189,7 +201,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 const uint32_t kf = smem_u32(&bars->k_full[s]);
                 mbar_expect_tx(kf, static_cast<uint32_t>(k_stage_bytes));
                 for (int a = 0; a < atoms; ++a)
-                    tma_load_2d(smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128), &tmap_k, a * atom_elems, (tile_begin + it) * TC_KEYS, kf);
+                    tma_load_2d(smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128), &tmap_k, a * atom_elems,
+                                static_cast<int>(key_base) + (tile_begin + it) * TC_KEYS, kf);
                 issued = it + 1;
             }
             if (*aborted) {   // let the copies already in flight land before the CTA leaves
@@ -201,7 +214,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_vis > 0) {
-            constexpr uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, TC_N);
+            constexpr uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N);   // ragged: only the first query row's heads
             bool ok = mbar_wait(smem_u32(&bars->q_full), 0);
             uint32_t cnt = 0;
             for (int it = 0; it < n_vis && ok; ++it) {
@@ -235,6 +248,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
     } else {
         // ------------------------------------------------------------------ epilogue: warps 2..9
+        constexpr int NCHUNK = RAGGED ? H / 32 : TC_N / 32;   // 32-column chunks to reduce (ragged: the first query row only)
+        static_assert(NCHUNK % 2 == 0, "chunks are processed in pairs");
         const int e = (warp - 2) >> 2;          // epilogue group = TMEM half it drains
         const int quad = warp & 3;              // TMEM lanes 32*quad .. 32*quad+31
         const float neg_inf = __int_as_float(0xff800000);
@@ -251,8 +266,9 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             __syncwarp();                                        // slots are free again
         };
         for (int it = 0; it < n_vis && ok; ++it) {
-            const int64_t s = static_cast<int64_t>(tile_begin + it) * TC_KEYS + quad * 32 + lane;
-            const bool key_ok = s < p.n_keys;
+            const int64_t s_local = static_cast<int64_t>(tile_begin + it) * TC_KEYS + quad * 32 + lane;
+            const bool key_ok = s_local < key_count;
+            const int64_t s = key_base + s_local;               // row of k_idx (and of k_scale / col_bias; ragged: of scores)
             const float kscale = (FP8 && key_ok) ? p.k_scale[s] : 1.f;
             const float cb = (p.col_bias != nullptr && key_ok) ? p.col_bias[s] : 0.f;
             for (int j = e; j < nq; j += 2) {
@@ -265,7 +281,13 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 auto store = [&](int tt, float v) {
                     const int t = tsub0 + tt;
-                    if constexpr (!CAND) {
+                    if constexpr (RAGGED) {
+                        if (tt == 0 && j == 0 && key_ok) {
+                            float out = v * kscale;
+                            out = fmaf(rbs[0], cb, out);
+                            p.scores[s] = out;
+                        }
+                    } else if constexpr (!CAND) {
                         if (t < p.M && key_ok) {
                             float out = v * kscale;
                             out = fmaf(rbs[j * TPS + tt], cb, out);
@@ -293,12 +315,12 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 uint32_t ra[32], rb[32];
                 tmem_ld32_issue(taddr, ra);
 #pragma unroll
-                for (int c = 0; c < TC_N / 32; c += 2) {
+                for (int c = 0; c < NCHUNK; c += 2) {
                     tmem_ld_wait(ra);
                     tmem_ld32_issue(taddr + (c + 1) * 32, rb);
                     reduce_chunk<H>(ra, ws + j * TC_N + c * 32, c * 32, acc, store);
                     tmem_ld_wait(rb);
-                    if (c + 2 < TC_N / 32) {
+                    if (c + 2 < NCHUNK) {
                         tmem_ld32_issue(taddr + (c + 2) * 32, ra);
                     } else {
                         // every column of this TMEM half is in registers: hand it back before the last reduction
@@ -318,7 +340,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             }
         }
         // key tiles no token of this CTA may see: -inf (score-matrix mode only)
-        for (int tile = vis_end + e; !CAND && tile < tile_end; tile += 2) {
+        for (int tile = vis_end + e; !CAND && !RAGGED && tile < tile_end; tile += 2) {
             const int64_t s = static_cast<int64_t>(tile) * TC_KEYS + quad * 32 + lane;
             if (s < p.n_keys)
                 for (int t = t0; t <= t_hi; ++t) p.scores[static_cast<int64_t>(t) * p.ld + s] = neg_inf;
@@ -373,11 +395,11 @@ bool indexer_tc_candidates_supported(int H, int D, int dtype) {
     return (H == 32 || H == 64) && (nq_max / 2) * (TC_N / H) <= TC_CAND_TPW;
 }
 
-template <int H, bool FP8, bool CAND>
+template <int H, bool FP8, bool CAND, bool RAGGED = false>
 static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, const TcCandParams& cp, dim3 grid, size_t smem,
                      cudaStream_t stream) {
-    JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8, CAND>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    indexer_tc_kernel<H, FP8, CAND><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p, cp);
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8, CAND, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    indexer_tc_kernel<H, FP8, CAND, RAGGED><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p, cp);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
@@ -392,7 +414,7 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
     p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = ld; p.n_keys = n_keys; p.q_pos0 = q_pos0;
     p.M = M; p.H = H; p.causal = causal; p.dev_status = dev_status;
-    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap};
+    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap, nullptr};
     p.atoms = D * esz / 128;
     p.nq = p.atoms == 1 ? 4 : 2;
     const int tps = TC_N / H;
@@ -442,6 +464,49 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     }
 #undef JANUS_TC_CASE
     return JANUS_ERR_UNSUPPORTED;
+}
+
+// Ragged batch (decode): B query rows, row b against keys key_offsets[b] .. key_offsets[b+1] of one concatenated array.
+bool indexer_tc_batch_supported(int B, int H, int D, int64_t total_keys, int dtype) {
+    const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
+    return H == 64 && (row_bytes == 128 || row_bytes == 256) && static_cast<int64_t>(B) * H < (int64_t(1) << 31) &&
+           total_keys < (int64_t(1) << 31) - 256 && B <= 65535;
+}
+
+int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stride_tok, const float* w, const float* q_scale,
+                            int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int B, int H, int D,
+                            int64_t total_keys, int64_t max_keys, const int64_t* key_offsets, int dtype, float* scores, int32_t* dev_status,
+                            cudaStream_t stream) {
+    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3;
+    const int esz = fp8 ? 1 : 2;
+    TcParams p;
+    p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
+    p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = 0; p.n_keys = total_keys; p.q_pos0 = 0;
+    p.M = B; p.H = H; p.causal = 0; p.dev_status = dev_status;
+    const TcCandParams cp{nullptr, nullptr, nullptr, 0, key_offsets};
+    p.atoms = D * esz / 128;
+    p.nq = 2;
+    const int tps = TC_N / H;
+    const int q_bytes = p.nq * p.atoms * TC_N * 128;
+    const int k_stage = p.atoms * TC_KEYS * 128;
+    const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + 2 * p.nq * tps) + static_cast<int>(sizeof(TcBarriers)) + 16;
+    p.stages = (TC_SMEM_BUDGET - q_bytes - tail) / k_stage;
+    if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
+    if (p.stages < 2) return JANUS_ERR_UNSUPPORTED;
+    const size_t smem = static_cast<size_t>(q_bytes) + static_cast<size_t>(p.stages) * k_stage + tail;
+    const int max_tiles = static_cast<int>((max_keys + TC_KEYS - 1) / TC_KEYS);
+    p.n_tiles = max_tiles;
+    int64_t per = (static_cast<int64_t>(max_tiles) * B + 148 * 4 - 1) / (148 * 4);
+    if (per < 2) per = 2;
+    if (per > 64) per = 64;
+    p.tiles_per_cta = static_cast<int>(per);
+    dim3 grid((max_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, B);
+    CUtensorMap tq, tk;
+    const uint32_t box_cols = fp8 ? 128 : 64;
+    if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(B) * H, D, static_cast<uint64_t>(D) * esz, TC_N, box_cols)) return JANUS_ERR_CUDA;
+    if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(total_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols))
+        return JANUS_ERR_CUDA;
+    return fp8 ? launch_tc<64, true, false, true>(tq, tk, p, cp, grid, smem, stream) : launch_tc<64, false, false, true>(tq, tk, p, cp, grid, smem, stream);
 }
 
 }  // namespace janus

@@ -135,6 +135,23 @@ page_lists_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restric
                         dev_status, scan_scratch);
 }
 
+// Batch form (decode over many sessions): row r of idx belongs to a session with its own page table
+// page_tables[table_offsets[r] .. table_offsets[r+1]) and its own history length demand_limits[r]; physical page ids are
+// global, so all rows mark one bitmap.  Sizes are small (rows x k indices), so this is the plain one-index-per-thread form.
+__global__ void __launch_bounds__(MARK_THREADS)
+page_mark_rows_kernel(const int32_t* __restrict__ idx, int64_t n_rows, int k, const int64_t* __restrict__ demand_limits, int page_size,
+                      int page_shift, const int32_t* __restrict__ page_tables, const int64_t* __restrict__ table_offsets,
+                      int64_t n_phys_pages, uint32_t* __restrict__ bitmap, int32_t* dev_status) {
+    const int64_t n_idx = n_rows * k;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * MARK_THREADS;
+    for (int64_t e = static_cast<int64_t>(blockIdx.x) * MARK_THREADS + threadIdx.x; e < n_idx; e += stride) {
+        const int64_t r = e / k;
+        const int64_t off = __ldg(table_offsets + r);
+        mark_one(__ldg(idx + e), __ldg(demand_limits + r), page_size, page_shift, page_tables + off, __ldg(table_offsets + r + 1) - off,
+                 n_phys_pages, bitmap, dev_status);
+    }
+}
+
 __global__ void page_union_kernel(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, int n_words) {
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += gridDim.x * blockDim.x) dst[i] |= src[i];
 }
@@ -189,6 +206,42 @@ extern "C" int janus_page_demand(const int32_t* idx, int64_t n_rows, int k, int6
         else
             page_mark_kernel<false><<<static_cast<unsigned>(blocks), MARK_THREADS, 0, stream>>>(
                 idx, n_idx, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bitmap, n_words, dev_status);
+        JANUS_CUDA_CHECK(cudaGetLastError());
+    }
+    page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs,
+                                                     miss_pages, n_miss, miss_runs, n_miss_runs, capacity, dev_status);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
+
+extern "C" int janus_page_demand_batch(const int32_t* idx, int64_t n_rows, int k, const int64_t* demand_limits, int page_size,
+                                       const int32_t* page_tables, const int64_t* table_offsets, int64_t n_phys_pages,
+                                       const uint32_t* predicted_bitmap, uint32_t* bitmap, int32_t* pages, int32_t* n_pages,
+                                       int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss, int32_t* miss_runs,
+                                       int32_t* n_miss_runs, int64_t capacity, int32_t* dev_status, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n_rows < 0 || k < 0 || page_size <= 0 || n_phys_pages <= 0 || capacity < 0) return JANUS_ERR_INVALID_ARG;
+    if (n_phys_pages > (int64_t(1) << 31) - 64) return JANUS_ERR_UNSUPPORTED;
+    if (!bitmap || !pages || !n_pages || !runs || !n_runs) return JANUS_ERR_INVALID_ARG;
+    const int n_miss_ptrs = (miss_pages != nullptr) + (n_miss != nullptr) + (miss_runs != nullptr) + (n_miss_runs != nullptr);
+    if (n_miss_ptrs != 0 && n_miss_ptrs != 4) return JANUS_ERR_INVALID_ARG;
+    const int64_t n_idx = n_rows * static_cast<int64_t>(k);
+    if (n_idx > 0 && (!idx || !demand_limits || !page_tables || !table_offsets)) return JANUS_ERR_INVALID_ARG;
+
+    const int n_words = static_cast<int>((n_phys_pages + 31) / 32);
+    JANUS_CUDA_CHECK(cudaMemsetAsync(bitmap, 0, sizeof(uint32_t) * n_words, stream));
+    if (n_idx > 0) {
+        int page_shift = -1;
+        if ((page_size & (page_size - 1)) == 0) {
+            page_shift = 0;
+            while ((1 << page_shift) < page_size) ++page_shift;
+        }
+        int64_t blocks = (n_idx + MARK_THREADS * 4 - 1) / (MARK_THREADS * 4);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        page_mark_rows_kernel<<<static_cast<unsigned>(blocks), MARK_THREADS, 0, stream>>>(idx, n_rows, k, demand_limits, page_size, page_shift,
+                                                                                          page_tables, table_offsets, n_phys_pages, bitmap,
+                                                                                          dev_status);
         JANUS_CUDA_CHECK(cudaGetLastError());
     }
     page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs,

@@ -16,8 +16,8 @@ __global__ void __launch_bounds__(AG_THREADS)
 sparse_attn_generic_kernel(const uint16_t* __restrict__ q, int M, int H_q, int d_qk, const uint16_t* __restrict__ k_pool,
                            const uint16_t* __restrict__ v_pool, int64_t page_stride, int64_t tok_stride, int64_t head_stride,
                            int n_kv_heads, int d_v, const int32_t* __restrict__ idx, int k, int page_size,
-                           const int32_t* __restrict__ page_table, int64_t n_logical_pages, float softmax_scale,
-                           uint16_t* __restrict__ out, float* __restrict__ lse, int32_t* dev_status) {
+                           const int32_t* __restrict__ page_table, int64_t n_logical_pages, const int64_t* __restrict__ table_offsets,
+                           float softmax_scale, uint16_t* __restrict__ out, float* __restrict__ lse, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int kpad = d_qk + 8, vpad = d_v + 8;             // row pitch in bf16: odd multiple of 16 bytes -> conflict-free 16 B reads
     const bool v_alias = (v_pool == k_pool);
@@ -31,6 +31,10 @@ sparse_attn_generic_kernel(const uint16_t* __restrict__ q, int M, int H_q, int d
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int t = blockIdx.x;
+    if (table_offsets != nullptr) {     // every row has a page table of its own (a batch of sessions)
+        page_table += table_offsets[t];
+        n_logical_pages = table_offsets[t + 1] - table_offsets[t];
+    }
     const int heads_per_kv = H_q / n_kv_heads;
     const int groups_per_kv = (heads_per_kv + G - 1) / G;
     const int hk = blockIdx.y / groups_per_kv;
@@ -158,8 +162,8 @@ sparse_attn_generic_kernel(const uint16_t* __restrict__ q, int M, int H_q, int d
 template <int G>
 static int launch_g(const void* q, int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
                     int64_t tok_stride, int64_t head_stride, int n_kv_heads, int d_v, const int32_t* idx, int k, int page_size,
-                    const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out, float* lse,
-                    int32_t* dev_status, cudaStream_t stream) {
+                    const int32_t* page_table, int64_t n_logical_pages, const int64_t* table_offsets, float softmax_scale, void* out,
+                    float* lse, int32_t* dev_status, cudaStream_t stream) {
     const bool v_alias = (v_pool == k_pool);
     size_t smem = sizeof(uint16_t) * AG_KT * (d_qk + 8) + (v_alias ? 0 : sizeof(uint16_t) * AG_KT * (d_v + 8)) +
                   sizeof(float) * (G * d_qk + G * AG_KT + G) + sizeof(int) * AG_KT;
@@ -168,19 +172,19 @@ static int launch_g(const void* q, int M, int H_q, int d_qk, const void* k_pool,
     dim3 grid(M, n_kv_heads * ((heads_per_kv + G - 1) / G));
     sparse_attn_generic_kernel<G><<<grid, AG_THREADS, smem, stream>>>(
         static_cast<const uint16_t*>(q), M, H_q, d_qk, static_cast<const uint16_t*>(k_pool), static_cast<const uint16_t*>(v_pool),
-        page_stride, tok_stride, head_stride, n_kv_heads, d_v, idx, k, page_size, page_table, n_logical_pages, softmax_scale,
-        static_cast<uint16_t*>(out), lse, dev_status);
+        page_stride, tok_stride, head_stride, n_kv_heads, d_v, idx, k, page_size, page_table, n_logical_pages, table_offsets,
+        softmax_scale, static_cast<uint16_t*>(out), lse, dev_status);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
 
 int launch_sparse_attn_generic(const void* q, int M, int H_q, int d_qk, const void* k_pool, const void* v_pool, int64_t page_stride,
                                int64_t tok_stride, int64_t head_stride, int n_kv_heads, int d_v, const int32_t* idx, int k,
-                               int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
-                               float* lse, int32_t* dev_status, cudaStream_t stream) {
+                               int page_size, const int32_t* page_table, int64_t n_logical_pages, const int64_t* table_offsets,
+                               float softmax_scale, void* out, float* lse, int32_t* dev_status, cudaStream_t stream) {
     const int heads_per_kv = H_q / n_kv_heads;
 #define JANUS_AG_ARGS q, M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, head_stride, n_kv_heads, d_v, idx, k, page_size, \
-                      page_table, n_logical_pages, softmax_scale, out, lse, dev_status, stream
+                      page_table, n_logical_pages, table_offsets, softmax_scale, out, lse, dev_status, stream
     if (heads_per_kv >= 8) return launch_g<8>(JANUS_AG_ARGS);
     if (heads_per_kv >= 4) return launch_g<4>(JANUS_AG_ARGS);
     if (heads_per_kv >= 2) return launch_g<2>(JANUS_AG_ARGS);

@@ -94,6 +94,7 @@ struct LpParams {
     int page_size, page_shift;
     const int32_t* page_table;
     int64_t n_logical_pages;
+    const int64_t* table_offsets;   // NULL, or [M + 1]: row t uses page_table[table_offsets[t] .. table_offsets[t + 1])
     float scale_log2e;        // softmax_scale * log2(e)
     uint16_t* out;
     float* lse;
@@ -284,22 +285,28 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         bool ok = true;
         LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
         const long long prof_t0 = LP_PROF_NOW();
+        int64_t tbl_nxt = 0, tbl_n_nxt = p.n_logical_pages;     // page table (start, length) of the query row the last load_raw was for
         auto load_raw = [&](int gh) -> int {                   // lane r owns row r of global half-tile gh
             if (gh >= total_half) return -1;
             const int it = gh / n_half;
             const int slot = (gh - it * n_half) * LP_HALF + lane;
-            return slot < p.k ? __ldg(p.idx + static_cast<int64_t>(cid + it * n_clusters) * p.k + slot) : -1;
+            const int64_t t_row = cid + it * n_clusters;
+            if (p.table_offsets != nullptr) {                  // every query row has a page table of its own (a batch of sessions)
+                tbl_nxt = __ldg(p.table_offsets + t_row);
+                tbl_n_nxt = __ldg(p.table_offsets + t_row + 1) - tbl_nxt;
+            }
+            return slot < p.k ? __ldg(p.idx + t_row * p.k + slot) : -1;
         };
-        auto resolve = [&](int s_tok, bool& valid) -> const unsigned char* {   // first owned byte of the row of token s_tok
+        auto resolve = [&](int s_tok, int64_t tbl, int64_t tbl_n, bool& valid) -> const unsigned char* {   // first owned byte of the row of token s_tok
             const unsigned char* ptr = reinterpret_cast<const unsigned char*>(p.pool) + seg_off;
             valid = false;
             if (s_tok >= 0) {
                 const int64_t lp = p.page_shift >= 0 ? (s_tok >> p.page_shift) : (s_tok / p.page_size);
                 const int within = p.page_shift >= 0 ? (s_tok & (p.page_size - 1)) : (s_tok % p.page_size);
-                if (lp >= p.n_logical_pages) {
+                if (lp >= tbl_n) {
                     report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
                 } else {
-                    ptr += (static_cast<int64_t>(__ldg(p.page_table + lp)) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
+                    ptr += (static_cast<int64_t>(__ldg(p.page_table + tbl + lp)) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
                     valid = true;
                 }
             }
@@ -311,7 +318,8 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             return gh;
         };
         bool valid_cur, valid_nxt = false;
-        const unsigned char* row_ptr = resolve(load_raw(g), valid_cur);
+        const int raw0 = load_raw(g);
+        const unsigned char* row_ptr = resolve(raw0, tbl_nxt, tbl_n_nxt, valid_cur);
         const unsigned char* row_nxt = row_ptr;
         int hi_nxt = next_owned(g);
         int raw_nxt = load_raw(hi_nxt);
@@ -344,7 +352,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                 }
             }
             cp_async_commit();
-            row_nxt = resolve(raw_nxt, valid_nxt);                 // page-table load overlaps the copies in flight
+            row_nxt = resolve(raw_nxt, tbl_nxt, tbl_n_nxt, valid_nxt);   // page-table load overlaps the copies in flight
             raw_nxt = load_raw(next_owned(hi_nxt));
             LP_PROF_WAIT(w_group, (cp_async_wait<0>(), true));
             fence_proxy_async();              // publish the landed rows to the MMA (async) proxy
@@ -652,8 +660,8 @@ bool sparse_attn_latent_tc_supported(int M, int H_q, int d_qk, const void* k_poo
 }
 
 int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t page_stride, int64_t tok_stride, const int32_t* idx, int k,
-                                 int page_size, const int32_t* page_table, int64_t n_logical_pages, float softmax_scale, void* out,
-                                 float* lse, int32_t* dev_status, cudaStream_t stream) {
+                                 int page_size, const int32_t* page_table, int64_t n_logical_pages, const int64_t* table_offsets,
+                                 float softmax_scale, void* out, float* lse, int32_t* dev_status, cudaStream_t stream) {
     LpParams p;
     p.q = static_cast<const uint16_t*>(q);
     p.pool = static_cast<const uint16_t*>(pool);
@@ -669,6 +677,7 @@ int launch_sparse_attn_latent_tc(const void* q, int M, const void* pool, int64_t
     }
     p.page_table = page_table;
     p.n_logical_pages = n_logical_pages;
+    p.table_offsets = table_offsets;
     p.scale_log2e = softmax_scale * 1.4426950408889634f;
     p.out = static_cast<uint16_t*>(out);
     p.lse = lse;

@@ -31,7 +31,39 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_
     topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix64), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh);
 }
 
+// Batch form (decode over many sessions): row b starts at scores[row_offsets[b]] and has row_lengths[b] elements (or runs
+// up to the next row's start when row_lengths is NULL), every element visible.
+template <int CAP>
+__global__ void __launch_bounds__(TK_THREADS)
+topk_ragged_kernel(const float* __restrict__ scores, const int64_t* __restrict__ row_offsets, const int64_t* __restrict__ row_lengths, int k,
+                   int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    using TopkShared = TopkSharedT<CAP>;
+    TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+    const int b = blockIdx.x;
+    const int64_t off = row_offsets[b];
+    int64_t n = row_lengths != nullptr ? row_lengths[b] : row_offsets[b + 1] - off;
+    if (n < 0) n = 0;
+    if (n > 2147483639) n = 2147483639;
+    topk_row(scores + off, static_cast<int>(n), k, b, idx + static_cast<int64_t>(b) * k, count, kth, sh);
+}
+
 }  // namespace janus
+
+extern "C" int janus_topk_batch(const float* scores, const int64_t* row_offsets, const int64_t* row_lengths, int B, int k, int32_t* idx,
+                                int32_t* count, float* kth, int32_t* /*dev_status*/, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (B < 0 || k <= 0) return JANUS_ERR_INVALID_ARG;
+    if (B == 0) return JANUS_OK;
+    if (!idx || !row_offsets || !scores || !aligned16(scores)) return JANUS_ERR_INVALID_ARG;
+    // row lengths live on the device: the large candidate buffer serves any length
+    const size_t smem = sizeof(TopkSharedT<TK_CAP>);
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_ragged_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    topk_ragged_kernel<TK_CAP><<<B, TK_THREADS, smem, stream>>>(scores, row_offsets, row_lengths, k, idx, count, kth);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
 
 extern "C" size_t janus_topk_workspace_size(int, int64_t, int) { return 0; }
 

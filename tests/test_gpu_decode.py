@@ -1,0 +1,116 @@
+"""Decode step over a batch of sessions (Sec. 2.2, "Decode phase": an append prefill with a single appended token per
+session) through the C ABI: janus_indexer_scores_batch -> janus_topk_batch -> janus_page_demand_batch ->
+janus_sparse_attn_decode, each checked against the oracle session by session.  Sessions have ragged history lengths
+(one shorter than k, one shorter than a key tile), their own page tables into one global KV pool, and concatenated
+indexer keys."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import janus_oracle as O
+from paper_2609_36938_b200 import binding as B
+from paper_2609_36938_b200 import build
+from paper_2609_36938_b200 import workloads as W
+
+import helpers as Hp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.load()
+    yield
+    B.check_dev_status()
+
+
+def make_batch(seed, lengths, dtype, H=64, D=128, page=64):
+    """Session b: L_b cached tokens plus the new one.  Keys are concatenated with rows padded to a multiple of 4."""
+    rng = np.random.default_rng(seed)
+    nb = len(lengths)
+    key_off = [0]
+    for L in lengths:
+        key_off.append(key_off[-1] + (L + 1 + 3) // 4 * 4)
+    total = key_off[-1]
+    kf = rng.standard_normal((total, D)).astype(np.float32)
+    qf = rng.standard_normal((nb, H, D)).astype(np.float32)
+    b = {"lengths": lengths, "key_off": np.array(key_off, np.int64), "w": (rng.uniform(0, 1, (nb, H)) / 8).astype(np.float32), "dtype": dtype,
+         "q_scale": None, "k_scale": None}
+    if dtype == "bf16":
+        b["q"], b["k"] = W.to_bf16_bits(qf), W.to_bf16_bits(kf)
+    else:
+        b["q"], b["k"] = W.to_e4m3_bits(2 * qf), W.to_e4m3_bits(2 * kf)
+        b["q_scale"] = np.exp2(rng.uniform(-2, 2, (nb, H))).astype(np.float32)
+        b["k_scale"] = np.exp2(rng.uniform(-1, 1, total)).astype(np.float32)
+    # page tables: session b needs ceil((L_b + 1) / page) pages, drawn without replacement from one global pool
+    n_pages = [(L + 1 + page - 1) // page for L in lengths]
+    n_phys = sum(n_pages) + 37
+    perm = rng.permutation(n_phys)
+    tab_off = np.concatenate([[0], np.cumsum(n_pages)]).astype(np.int64)
+    b["tables"] = perm[:tab_off[-1]].astype(np.int32)
+    b["tab_off"], b["n_phys"], b["page"] = tab_off, n_phys, page
+    return b
+
+
+def session_keys(b, i):
+    a = int(b["key_off"][i])
+    return slice(a, a + b["lengths"][i] + 1)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_decode_batch_matches_oracle_session_by_session(dtype):
+    lengths = [5000, 12345, 300, 20000, 40, 7777, 129]
+    k, page, d_qk, d_v, H_q = 128, 64, 576, 512, 128
+    b = make_batch(11, lengths, dtype, page=page)
+    nb = len(lengths)
+    rng = np.random.default_rng(5)
+    q_attn = W.to_bf16_bits((rng.standard_normal((nb, H_q, d_qk)) / 4).astype(np.float32))
+    pool = W.to_bf16_bits((rng.standard_normal((b["n_phys"], page, 1, d_qk)) / 4).astype(np.float32))
+    scale = 1.0 / np.sqrt(d_qk)
+
+    dev = lambda x, kind: B.to_device(x, kind)
+    key_off = torch.from_numpy(b["key_off"]).cuda()
+    tab_off = torch.from_numpy(b["tab_off"]).cuda()
+    limits = torch.tensor(lengths, dtype=torch.int64, device="cuda")
+    kd = dev(b["k"], dtype)
+
+    # ---- indexer
+    # key_offsets[b+1] - key_offsets[b] includes the padding rows: they are scored like keys (their bits are whatever the
+    # caller put there) and left out of the selection through row_lengths
+    scores = B.janus_indexer_scores_batch(dev(b["q"], dtype), kd, dev(b["w"], "f32"), key_off, max(lengths) + 4,
+                                          q_scale=dev(b["q_scale"], "f32"), k_scale=dev(b["k_scale"], "f32"))
+    row_len = torch.tensor([L + 1 for L in lengths], dtype=torch.int64, device="cuda")
+    idx, cnt, kth = B.janus_topk_batch(scores, key_off, k, row_lengths=row_len)
+    pd = B.janus_page_demand_batch(idx, demand_limits=limits, page_size=page, page_tables=dev(b["tables"], "i32"), table_offsets=tab_off,
+                                   n_phys_pages=b["n_phys"])
+    out, lse = B.janus_sparse_attn_decode(dev(q_attn, "bf16"), dev(pool, "bf16"), dev(pool, "bf16"), idx, page_tables=dev(b["tables"], "i32"),
+                                          table_offsets=tab_off, page_size=page, softmax_scale=scale, d_v=d_v)
+    B.check_dev_status()
+    scores_h, idx_h, cnt_h = scores.cpu().numpy(), idx.cpu().numpy(), cnt.cpu().numpy()
+    out_h, lse_h = Hp.bf16_tensor_to_f64(out), lse.cpu().numpy().astype(np.float64)
+
+    all_pages = set()
+    for i, L in enumerate(lengths):
+        ks = session_keys(b, i)
+        ref = O.indexer_scores(b["q"][i:i + 1], b["k"][ks], b["w"][i:i + 1], dtype=dtype,
+                               q_scale=None if b["q_scale"] is None else b["q_scale"][i:i + 1],
+                               k_scale=None if b["k_scale"] is None else b["k_scale"][ks], q_pos0=L, causal=True)
+        Hp.assert_scores_close(scores_h[ks][None, :], ref, 1e-4 if dtype == "bf16" else 1e-4, f"session {i} scores")
+        # selection over the session's L + 1 keys
+        n_sel = min(k, L + 1)
+        assert cnt_h[i] == n_sel and idx_h[i].max() <= L
+        ok, msg = O.topk_row_agrees(idx_h[i], ref[0], L + 1, k)
+        assert ok, f"session {i}: {msg}"
+        # pages of the selected history tokens through the session's own table
+        table = b["tables"][b["tab_off"][i]:b["tab_off"][i + 1]]
+        all_pages |= set(O.page_demand(idx_h[i:i + 1], L, page, table)["pages"])
+        # attention of the one query row over its selection
+        ref_o, ref_lse = O.sparse_attention(q_attn[i:i + 1], pool, pool, table, idx_h[i:i + 1], page_size=page, softmax_scale=scale,
+                                            d_qk=d_qk, d_v=d_v)
+        Hp.assert_attention_close(out_h[i:i + 1], ref_o, f"session {i} attention")
+        np.testing.assert_allclose(lse_h[i:i + 1], ref_lse, rtol=2e-3, atol=2e-3)
+    got = Hp.page_lists_from_device(pd)
+    assert got["pages"] == sorted(all_pages)
+    assert got["runs"] == [tuple(r) for r in O.maximal_runs(sorted(all_pages))]
+    assert got["miss"] == sorted(all_pages)          # nothing declared resident
