@@ -153,6 +153,74 @@ def run_reference(args, shp, sess):
                       f"rows are independent, rows/s reported as tokens/s", "ms_per_step": dt * 1e3}
 
 
+def run_decode(args):
+    """Side workload (not the headline metric): one decode step over `--decode-batch` sessions of `--L` cached tokens each
+    (default 131072), FP8 64 x 128 indexer, latent attention, k = 2048.  Inputs are made on the device (parity of this
+    path is covered by tests/test_gpu_decode.py); prints one JSON line with per-call times and the indexer's bandwidth."""
+    import torch
+    from paper_2609_36938_b200 import binding as B, build as _build
+
+    torch.cuda.set_device(0)
+    _build.build()
+    B.load()
+    nb, L, k, page, H, D = args.decode_batch, (args.L or 131072), 2048, 64, 64, 128
+    g = torch.Generator(device="cuda").manual_seed(args.seed)
+    n_keys = (L + 1 + 3) // 4 * 4
+    key_off = torch.arange(nb + 1, dtype=torch.int64, device="cuda") * n_keys
+    row_len = torch.full((nb,), L + 1, dtype=torch.int64, device="cuda")
+    k_idx = torch.randint(0, 256, (nb * n_keys, D), dtype=torch.uint8, device="cuda", generator=g)
+    k_idx = torch.where((k_idx & 0x7f) >= 0x7f, k_idx & 0xf7, k_idx)          # no NaN codes
+    q_idx = torch.randint(0, 120, (nb, H, D), dtype=torch.uint8, device="cuda", generator=g)
+    w = torch.rand((nb, H), device="cuda", generator=g) / 8
+    q_scale = torch.ones((nb, H), device="cuda") / 64
+    k_scale = torch.ones((nb * n_keys,), device="cuda") / 64
+    pages_per = (L + 1 + page - 1) // page
+    n_phys = nb * pages_per
+    tables = torch.randperm(n_phys, device="cuda", generator=g).int()
+    tab_off = torch.arange(nb + 1, dtype=torch.int64, device="cuda") * pages_per
+    limits = torch.full((nb,), L, dtype=torch.int64, device="cuda")
+    pool = (torch.randn((n_phys, page, 1, 576), device="cuda", generator=g) / 24).bfloat16()
+    q = (torch.randn((nb, 128, 576), device="cuda", generator=g) / 24).bfloat16()
+    scores = torch.empty((nb * n_keys,), dtype=torch.float32, device="cuda")
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        if marks: marks[0].record()
+        B.janus_indexer_scores_batch(q_idx, k_idx, w, key_off, n_keys, q_scale=q_scale, k_scale=k_scale, scores=scores)
+        if marks: marks[1].record()
+        idx, _, _ = B.janus_topk_batch(scores, key_off, k, row_lengths=row_len, want_count=False, want_kth=False)
+        if marks: marks[2].record()
+        pd = B.janus_page_demand_batch(idx, demand_limits=limits, page_size=page, page_tables=tables, table_offsets=tab_off, n_phys_pages=n_phys)
+        if marks: marks[3].record()
+        out, _ = B.janus_sparse_attn_decode(q, pool, pool, idx, page_tables=tables, table_offsets=tab_off, page_size=page,
+                                            softmax_scale=1 / 24, d_v=512, want_lse=False)
+        if marks: marks[4].record()
+        return out
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    B.check_dev_status()
+    marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for m in marks:
+        step(m)
+    torch.cuda.synchronize()
+    B.check_dev_status()
+    per = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks]).mean(axis=0)
+    total_ms = float(np.mean([m[0].elapsed_time(m[4]) for m in marks]))
+    peaks = load_peaks()
+    key_bytes = nb * (L + 1) * (D + 4 + 4)                    # key row + its scale read, score written
+    line = {"metric": "decode_tokens_per_sec_per_sparse_layer", "value": nb / (total_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+            "steps": args.steps, "ms_per_step": total_ms, "data": "synthetic (device-generated)", "dtype": "fp8_e4m3+bf16",
+            "config": {"workload": f"decode step: {nb} sessions x {L} cached tokens, k={k}, FP8 64x128 indexer, latent attention, page {page}"},
+            "kernels": {"indexer_scores_batch": {"ms": float(per[0]), "gbs": key_bytes / (per[0] * 1e-3) / 1e9,
+                                                 "frac_hbm_peak": key_bytes / (per[0] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                        "topk_batch": {"ms": float(per[1]), "gbs": nb * (L + 1) * 4 / (per[1] * 1e-3) / 1e9},
+                        "page_demand_batch": {"ms": float(per[2])},
+                        "sparse_attn_decode": {"ms": float(per[3]), "logical_gbs": nb * k * 1152 / (per[3] * 1e-3) / 1e9}}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -167,7 +235,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the side measurement of janus_indexer_topk")
+    ap.add_argument("--decode-batch", type=int, default=0, help="side workload: time one decode step over this many sessions instead")
     args = ap.parse_args()
+    if args.decode_batch > 0:
+        run_decode(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     args.steps_ref = max(1, min(args.steps, 3))
     args.warmup_ref = 1 if args.warmup > 0 else 0

@@ -223,6 +223,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars->k_full[s]), ph) && !*aborted;
                 if (!ok) break;
                 tc_fence_after();
+                // ragged mode has one query sub-tile, so consecutive key tiles alternate between the two TMEM halves
                 for (int j = 0; j < nq; ++j, ++cnt) {
                     const uint32_t slot = cnt & 1u, use = cnt >> 1;
                     ok = mbar_wait(smem_u32(&bars->tmem_empty[slot]), (use & 1u) ^ 1u) && !*aborted;
@@ -271,7 +272,9 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const int64_t s = key_base + s_local;               // row of k_idx (and of k_scale / col_bias; ragged: of scores)
             const float kscale = (FP8 && key_ok) ? p.k_scale[s] : 1.f;
             const float cb = (p.col_bias != nullptr && key_ok) ? p.col_bias[s] : 0.f;
-            for (int j = e; j < nq; j += 2) {
+            // score-matrix and candidate modes: group e drains the sub-tiles j = e, e+2, .. of every key tile (nq is even);
+            // ragged mode (nq = 1): group e drains the key tiles it = e, e+2, ..
+            for (int j = RAGGED ? ((it & 1) == e ? 0 : nq) : e; j < nq; j += 2) {
                 const uint32_t use = static_cast<uint32_t>(it * nq + j) >> 1;
                 ok = mbar_wait(smem_u32(&bars->tmem_full[e]), use & 1u) && !*aborted;
                 if (!ok) break;
@@ -485,7 +488,7 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
     p.M = B; p.H = H; p.causal = 0; p.dev_status = dev_status;
     const TcCandParams cp{nullptr, nullptr, nullptr, 0, key_offsets};
     p.atoms = D * esz / 128;
-    p.nq = 2;
+    p.nq = 1;
     const int tps = TC_N / H;
     const int q_bytes = p.nq * p.atoms * TC_N * 128;
     const int k_stage = p.atoms * TC_KEYS * 128;
