@@ -11,6 +11,7 @@
  *   - every data pointer is a DEVICE pointer owned by the caller, unless a comment says "host".
  *     The library never allocates or frees device memory; scratch, where a call needs it, is the
  *     caller's `ws` buffer of at least janus_<fn>_workspace_size(...) bytes (may be NULL when 0).
+ *     (janus_indexer_topk_static alone brings its own scratch: a fixed array in the library's device image.)
  *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
  *   - host-detectable problems (NULL pointer, bad size, misalignment, unsupported shape) return an
  *     error code and launch nothing.
