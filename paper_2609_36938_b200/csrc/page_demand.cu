@@ -135,6 +135,98 @@ page_lists_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restric
                         dev_status, scan_scratch);
 }
 
+// Large pools (a decode batch addresses the whole KV pool: 10^5 pages and more): the same lists built by one CTA per
+// 1024-word chunk.  A CTA first counts the ids / run starts / run ends of all words before its chunk (a few KB of bitmap
+// for the sizes this path is used for), then writes its part exactly like the single-CTA kernel; run lengths need every
+// start and end, so a small second kernel turns (start, end+1) into (start, length).  blockIdx.y = 0: the set itself,
+// 1: the miss set (bitmap AND NOT predicted).
+constexpr int LIST_MAX_CHUNKS = 64;
+
+__global__ void __launch_bounds__(LIST_THREADS)
+page_lists_chunk_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ predicted, int n_words, int64_t n_phys_pages,
+                        int32_t* pages, int32_t* n_pages, int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss,
+                        int32_t* miss_runs, int32_t* n_miss_runs, int64_t capacity, int32_t* dev_status) {
+    __shared__ int scan_scratch[40];
+    const bool miss = blockIdx.y == 1;
+    const uint32_t* a = bitmap;
+    const uint32_t* not_b = miss ? predicted : nullptr;
+    int32_t* ids = miss ? miss_pages : pages;
+    int32_t* n_ids = miss ? n_miss : n_pages;
+    int32_t* out_runs = miss ? miss_runs : runs;
+    int32_t* out_n_runs = miss ? n_miss_runs : n_runs;
+    auto word_at = [&](int i) -> uint32_t {
+        if (i < 0 || i >= n_words) return 0u;
+        uint32_t v = a[i];
+        if (not_b != nullptr) v &= ~not_b[i];
+        if (i == n_words - 1 && (n_phys_pages & 31)) v &= (1u << (n_phys_pages & 31)) - 1u;
+        return v;
+    };
+    auto starts_of = [&](int i, uint32_t v) { return v & ~((v << 1) | (word_at(i - 1) >> 31)); };
+    auto ends_of = [&](int i, uint32_t v) { return v & ~((v >> 1) | ((word_at(i + 1) & 1u) << 31)); };
+    const int base = blockIdx.x * LIST_THREADS;
+    // ---- everything before this chunk
+    int c_id = 0, c_st = 0, c_en = 0;
+    for (int i = threadIdx.x; i < base; i += LIST_THREADS) {
+        const uint32_t v = word_at(i);
+        c_id += __popc(v);
+        c_st += __popc(starts_of(i, v));
+        c_en += __popc(ends_of(i, v));
+    }
+    int id_base, run_base, end_base, dummy;
+    dummy = block_exclusive_scan<LIST_THREADS>(c_id, scan_scratch, &id_base);
+    dummy = block_exclusive_scan<LIST_THREADS>(c_st, scan_scratch, &run_base);
+    dummy = block_exclusive_scan<LIST_THREADS>(c_en, scan_scratch, &end_base);
+    (void)dummy;
+    // ---- this chunk
+    const int i = base + threadIdx.x;
+    const uint32_t v = word_at(i);
+    const uint32_t starts = starts_of(i, v), ends = ends_of(i, v);
+    int tot_ids, tot_starts, tot_ends;
+    int o_id = block_exclusive_scan<LIST_THREADS>(__popc(v), scan_scratch, &tot_ids) + id_base;
+    int o_st = block_exclusive_scan<LIST_THREADS>(__popc(starts), scan_scratch, &tot_starts) + run_base;
+    int o_en = block_exclusive_scan<LIST_THREADS>(__popc(ends), scan_scratch, &tot_ends) + end_base;
+    uint32_t m = v;
+    while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (o_id < capacity) ids[o_id] = i * 32 + b;
+        ++o_id;
+    }
+    m = starts;
+    while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (o_st < capacity) out_runs[2 * o_st] = i * 32 + b;
+        ++o_st;
+    }
+    m = ends;
+    while (m) {  // the j-th end closes the j-th start; end+1 is stored and turned into a length by the second kernel
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (o_en < capacity) out_runs[2 * o_en + 1] = i * 32 + b + 1;
+        ++o_en;
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
+        const int total_ids = id_base + tot_ids, total_runs = run_base + tot_starts;
+        *n_ids = total_ids;
+        *out_n_runs = total_runs;
+        if (total_ids > capacity || total_runs > capacity) report(dev_status, JANUS_DEV_CAPACITY_EXCEEDED);
+    }
+}
+
+__global__ void page_run_lengths_kernel(int32_t* runs, const int32_t* n_runs, int32_t* miss_runs, const int32_t* n_miss_runs, int64_t capacity) {
+    int32_t* r = blockIdx.y == 1 ? miss_runs : runs;
+    int64_t n = blockIdx.y == 1 ? *n_miss_runs : *n_runs;
+    if (n > capacity) n = capacity;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        r[2 * j + 1] -= r[2 * j];
+}
+
+// Chooses between the one-CTA list kernel (small bitmaps: one launch, no second pass) and the chunked pair.
+static int launch_page_lists(const uint32_t* bitmap, const uint32_t* predicted, int n_words, int64_t n_phys_pages, int32_t* pages,
+                             int32_t* n_pages, int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss, int32_t* miss_runs,
+                             int32_t* n_miss_runs, int64_t capacity, int32_t* dev_status, cudaStream_t stream);
+
 // Batch form (decode over many sessions): row r of idx belongs to a session with its own page table
 // page_tables[table_offsets[r] .. table_offsets[r+1]) and its own history length demand_limits[r]; physical page ids are
 // global, so all rows mark one bitmap.  Sizes are small (rows x k indices), so this is the plain one-index-per-thread form.
@@ -150,6 +242,25 @@ page_mark_rows_kernel(const int32_t* __restrict__ idx, int64_t n_rows, int k, co
         mark_one(__ldg(idx + e), __ldg(demand_limits + r), page_size, page_shift, page_tables + off, __ldg(table_offsets + r + 1) - off,
                  n_phys_pages, bitmap, dev_status);
     }
+}
+
+static int launch_page_lists(const uint32_t* bitmap, const uint32_t* predicted, int n_words, int64_t n_phys_pages, int32_t* pages,
+                             int32_t* n_pages, int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss, int32_t* miss_runs,
+                             int32_t* n_miss_runs, int64_t capacity, int32_t* dev_status, cudaStream_t stream) {
+    const int n_chunks = (n_words + LIST_THREADS - 1) / LIST_THREADS;
+    if (n_chunks >= 2 && n_chunks <= LIST_MAX_CHUNKS) {
+        const dim3 grid(n_chunks, miss_pages != nullptr ? 2 : 1);
+        page_lists_chunk_kernel<<<grid, LIST_THREADS, 0, stream>>>(bitmap, predicted, n_words, n_phys_pages, pages, n_pages, runs, n_runs, miss_pages,
+                                                                   n_miss, miss_runs, n_miss_runs, capacity, dev_status);
+        JANUS_CUDA_CHECK(cudaGetLastError());
+        page_run_lengths_kernel<<<dim3(64, grid.y), 256, 0, stream>>>(runs, n_runs, miss_runs, n_miss_runs, capacity);
+        JANUS_CUDA_CHECK(cudaGetLastError());
+        return JANUS_OK;
+    }
+    page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted, n_words, n_phys_pages, pages, n_pages, runs, n_runs, miss_pages, n_miss,
+                                                     miss_runs, n_miss_runs, capacity, dev_status);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
 }
 
 __global__ void page_union_kernel(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, int n_words) {
@@ -208,10 +319,8 @@ extern "C" int janus_page_demand(const int32_t* idx, int64_t n_rows, int k, int6
                 idx, n_idx, demand_limit, page_size, page_shift, page_table, n_logical_pages, n_phys_pages, bitmap, n_words, dev_status);
         JANUS_CUDA_CHECK(cudaGetLastError());
     }
-    page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs,
-                                                     miss_pages, n_miss, miss_runs, n_miss_runs, capacity, dev_status);
-    JANUS_CUDA_CHECK(cudaGetLastError());
-    return JANUS_OK;
+    return launch_page_lists(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs, miss_pages, n_miss, miss_runs,
+                             n_miss_runs, capacity, dev_status, stream);
 }
 
 extern "C" int janus_page_demand_batch(const int32_t* idx, int64_t n_rows, int k, const int64_t* demand_limits, int page_size,
@@ -244,8 +353,6 @@ extern "C" int janus_page_demand_batch(const int32_t* idx, int64_t n_rows, int k
                                                                                           dev_status);
         JANUS_CUDA_CHECK(cudaGetLastError());
     }
-    page_lists_kernel<<<1, LIST_THREADS, 0, stream>>>(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs,
-                                                     miss_pages, n_miss, miss_runs, n_miss_runs, capacity, dev_status);
-    JANUS_CUDA_CHECK(cudaGetLastError());
-    return JANUS_OK;
+    return launch_page_lists(bitmap, predicted_bitmap, n_words, n_phys_pages, pages, n_pages, runs, n_runs, miss_pages, n_miss, miss_runs,
+                             n_miss_runs, capacity, dev_status, stream);
 }

@@ -116,6 +116,29 @@ def test_page_demand_large_pool_uses_global_bitmap_and_reports_conditions():
         B.check_dev_status()
 
 
+def test_page_demand_chunked_lists_long_runs_and_miss_set():
+    # a pool large enough for the list kernel that works in 1024-word chunks (32768 pages each): one run of adjacent pages
+    # crosses word and chunk boundaries, scattered pages follow, and the miss set is taken against a predicted half
+    rng = np.random.default_rng(21)
+    pg, n_phys = 16, 110000
+    table = np.arange(n_phys, dtype=np.int32)                      # identity: physical adjacency = logical adjacency
+    run = np.arange(100, 70000)                                      # pages 100 .. 69999, crosses pages 32768 and 65536
+    scattered = rng.choice(np.arange(70010, n_phys), size=3000, replace=False)
+    pages_sel = np.concatenate([run, scattered])
+    toks = pages_sel * pg + rng.integers(0, pg, size=pages_sel.size)
+    pad = (-toks.size) % 128
+    idx = np.concatenate([toks, np.full(pad, -1)]).astype(np.int32).reshape(-1, 128)
+    rng.shuffle(idx, axis=0)
+    pred_pages = np.concatenate([run[::2], scattered[: 1500]])
+    pred = np.concatenate([pred_pages * pg, np.full((-pred_pages.size) % 64, -1)]).astype(np.int32).reshape(-1, 64)
+    got, ref, out = _run_page_demand(idx, n_phys * pg, pg, table, n_phys, pred_idx_np=pred)
+    B.check_dev_status()
+    assert got["pages"] == ref["pages"] and len(got["pages"]) == pages_sel.size
+    assert got["runs"] == ref["runs"] and got["runs"][0] == (100, 69900)
+    assert got["miss"] == ref["miss"]
+    assert got["miss_runs"] == ref["miss_runs"]
+
+
 def test_page_demand_is_deterministic():
     rng = np.random.default_rng(6)
     table = rng.permutation(2112).astype(np.int32)
