@@ -106,7 +106,7 @@ def captured_traffic(kernel_key: str, rows: int):
 
 
 def workload_numbers(shp):
-    """Algorithmic work of one step (exact pass), per the definitions in the design doc."""
+    """Algorithmic work of one step (exact pass): flops and bytes each call must do at least, from the shapes alone."""
     L, M, S = shp.L, shp.M, shp.S
     pairs = M * L + M * (M + 1) // 2
     sel = sum(min(shp.k, L + t + 1) for t in range(M))
