@@ -74,7 +74,7 @@ struct TcBarriers {
     int aborted;
 };
 
-// One 32-column chunk of accumulators: ReLU, weight, reduce over heads; a token's sum is complete every H columns.
+// One 32-column chunk of accumulators: 2 * ReLU, half weight, reduce over heads; a token's sum is complete every H columns.
 // Pairs of columns go through packed fp32 FMAs into up to four independent accumulator pairs, so the reduction is
 // neither one long dependent chain nor one instruction per element.
 template <int H, class Store>
@@ -88,7 +88,11 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
             const int i = 4 * i4 + 2 * j;                      // first column of the pair inside the chunk
             const int col = col0 + i;
             const float2 w2 = j == 0 ? make_float2(wv.x, wv.y) : make_float2(wv.z, wv.w);
-            const float2 x2 = make_float2(fmaxf(__uint_as_float(r[i]), 0.f), fmaxf(__uint_as_float(r[i + 1]), 0.f));
+            // 2 * max(x, 0) = x + |x|, exactly: an add (full-rate FMA pipe, |x| is an operand modifier) instead of a max (the
+            // half-rate pipe, which 256 of them per thread and tile would saturate before the tensor pipe); the weights
+            // carry the factor 1/2
+            const float xa = __uint_as_float(r[i]), xb = __uint_as_float(r[i + 1]);
+            const float2 x2 = make_float2(xa + fabsf(xa), xb + fabsf(xb));
             float2& a = acc[(col / 2) % NACC];
             a = ffma2(w2, x2, a);
             if (((col + 2) % H) == 0) {
@@ -172,7 +176,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             v = p.w[static_cast<int64_t>(t) * H + h];
             if (FP8) v *= p.q_scale[static_cast<int64_t>(t) * p.q_scale_stride_tok + h];
         }
-        ws[n] = v;
+        ws[n] = 0.5f * v;      // the epilogue forms 2 * relu
     }
     for (int n = threadIdx.x; n < tpc; n += TC_THREADS) {
         rbs[n] = (p.row_bias != nullptr && t0 + n < p.M) ? p.row_bias[t0 + n] : 0.f;
