@@ -150,6 +150,48 @@ def topk(scores, k: int, *, q_pos0: int = 0, causal: bool = True, rows=None) -> 
     return out
 
 
+# ----------------------------------------------------------------------------
+# entry granularity (footnote of Sec. 2.2: selection and attention per entry = a region of E consecutive tokens)
+# ----------------------------------------------------------------------------
+# The paper does not define how an entry is scored or masked.  Reading used here: the indexer has one key per entry, so
+# entry scores come from the same indexer run over entry keys; the query at position pos may select every entry that holds
+# at least one token at or before pos (entries 0 .. pos // E), and attends to the tokens of the selected entries that are at
+# or before pos.
+def entry_visible_prefix(t: int, n_entries: int, q_pos0: int, entry_size: int) -> int:
+    """Number of entries the query row t (position q_pos0 + t) may select."""
+    return max(0, min(n_entries, (q_pos0 + t) // entry_size + 1))
+
+
+def entry_topk(entry_scores, k_e: int, *, q_pos0: int, entry_size: int) -> np.ndarray:
+    """Row-wise top-k_e over entries.  Returns int64 [n_rows, k_e] padded with -1."""
+    entry_scores = np.asarray(entry_scores)
+    n_rows, n_entries = entry_scores.shape
+    out = np.full((n_rows, k_e), -1, dtype=np.int64)
+    for t in range(n_rows):
+        sel, _ = topk_select(entry_scores[t], entry_visible_prefix(t, n_entries, q_pos0, entry_size), k_e)
+        out[t, :len(sel)] = sel
+    return out
+
+
+def entry_expand(entry_idx, *, q_pos0: int, entry_size: int) -> np.ndarray:
+    """Token selection of entry selections: slot e*E + j of row t holds token entry_idx[t, e]*E + j if that token is at or
+    before position q_pos0 + t, else -1.  Returns int64 [n_rows, k_e * E]."""
+    entry_idx = np.asarray(entry_idx)
+    n_rows, k_e = entry_idx.shape
+    out = np.full((n_rows, k_e * entry_size), -1, dtype=np.int64)
+    for t in range(n_rows):
+        pos = q_pos0 + t
+        for e in range(k_e):
+            ent = int(entry_idx[t, e])
+            if ent < 0:
+                continue
+            for j in range(entry_size):
+                tok = ent * entry_size + j
+                if tok <= pos:
+                    out[t, e * entry_size + j] = tok
+    return out
+
+
 def topk_row_agrees(got_idx, score_row, prefix: int, k: int, band_rel: float = 1e-3):
     """Acceptance rule for one row of a selection computed elsewhere.
 

@@ -410,3 +410,29 @@ def test_workload_shapes_and_determinism():
     tabs, n_phys = W.fragmented_page_tables(shapes[:3], 0)
     allp = np.concatenate(tabs)
     assert len(np.unique(allp)) == len(allp) == n_phys
+
+
+# ---- entry granularity ------------------------------------------------------------------------------------------------
+def test_entry_selection_of_all_entries_expands_to_the_causal_prefix():
+    # selecting every visible entry must give exactly the tokens 0 .. pos of each row (so that attention over the expansion
+    # is dense causal attention), whatever the entry size and wherever the row sits inside its entry
+    for E, L, M in ((4, 10, 7), (8, 16, 9), (3, 0, 5), (16, 5, 3)):
+        n_entries = (L + M + E - 1) // E
+        scores = np.random.default_rng(E).standard_normal((M, n_entries))
+        sel = O.entry_topk(scores, n_entries, q_pos0=L, entry_size=E)
+        tok = O.entry_expand(sel, q_pos0=L, entry_size=E)
+        for t in range(M):
+            assert sorted(x for x in tok[t] if x >= 0) == list(range(L + t + 1))
+            assert O.entry_visible_prefix(t, n_entries, L, E) == (L + t) // E + 1
+
+
+def test_entry_topk_hand_case_and_unit_entries():
+    # E = 1 is token granularity: same selection as the token top-k
+    rng = np.random.default_rng(9)
+    sc = rng.standard_normal((6, 30))
+    assert np.array_equal(O.entry_topk(sc, 5, q_pos0=20, entry_size=1), O.topk(sc, 5, q_pos0=20, causal=True))
+    # hand case: E = 4, query at position 9 sees entries 0, 1, 2 (tokens 0..9); the best two of [0.5, 2.0, 1.0, 9.0] among
+    # the visible three are entries 1 and 2; their expansion drops tokens 10, 11 of entry 2
+    sel = O.entry_topk(np.array([[0.5, 2.0, 1.0, 9.0]]), 2, q_pos0=9, entry_size=4)
+    assert sel.tolist() == [[1, 2]]
+    assert O.entry_expand(sel, q_pos0=9, entry_size=4).tolist() == [[4, 5, 6, 7, 8, 9, -1, -1]]
