@@ -236,6 +236,26 @@ int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk,
                               void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * Entry granularity - selection and attention per entry, a region of `entry_size` consecutive tokens (footnote of
+ * Sec. 2.2; the paper does not define the entry-level scoring or masking, this library's reading is stated here).
+ * The indexer has one key per entry: entry scores are janus_indexer_scores over the entry keys with causal = 0.
+ *
+ *   janus_topk_entries   janus_topk over entries: row t (position q_pos0 + t) may select the entries that hold a token at
+ *                        or before its position, i.e. entries 0 .. (q_pos0 + t) / entry_size.  scores [M, scores_ld] fp32.
+ *   janus_entry_expand   idx_tokens[t, e * entry_size + j] = idx_entries[t, e] * entry_size + j if that token is at or
+ *                        before position q_pos0 + t, else -1 ([M, k_e * entry_size] int32).  The result feeds
+ *                        janus_page_demand and janus_sparse_attn_prefill like any token selection.
+ *
+ * A selection shared by a group of layers (index reuse) needs no call of its own: pass the same idx to the attention of
+ * every layer of the group.
+ */
+int janus_topk_entries(const float* scores, int64_t scores_ld, int M, int64_t n_entries,
+                       int64_t q_pos0, int entry_size, int k,
+                       int32_t* idx, int32_t* count, float* kth, int32_t* dev_status, void* stream);
+int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_size, int64_t q_pos0,
+                       int32_t* idx_tokens, void* stream);
+
+/*
  * Decode step over a batch of sessions (Sec. 2.2, "Decode phase"): one new token per session, processed like an append
  * prefill with a single appended token.  Session b has its own history, so the per-session arrays are concatenated and
  * addressed through offsets held in device memory:

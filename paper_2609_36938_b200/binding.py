@@ -29,6 +29,7 @@ EXPORTS = [
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
     "janus_indexer_scores_batch", "janus_topk_batch", "janus_page_demand_batch", "janus_sparse_attn_decode",
+    "janus_topk_entries", "janus_entry_expand",
 ]
 
 
@@ -89,6 +90,10 @@ def load() -> ctypes.CDLL:
     lib.janus_sparse_attn_decode.restype = c_i
     lib.janus_sparse_attn_decode.argtypes = [c_p, c_i, c_i, c_i, c_p, c_p, c_i64, c_i64, c_i64, c_i, c_i, c_p, c_i, c_i, c_p, c_p, c_f, c_p, c_p,
                                              c_p, c_p]
+    lib.janus_topk_entries.restype = c_i
+    lib.janus_topk_entries.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_p]
+    lib.janus_entry_expand.restype = c_i
+    lib.janus_entry_expand.argtypes = [c_p, c_i, c_i, c_i, c_i64, c_p, c_p]
     _lib = lib
     return lib
 
@@ -292,6 +297,31 @@ def janus_sparse_attn_prefill(q: torch.Tensor, k_pool: torch.Tensor, v_pool: tor
                                        _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_sparse_attn_prefill")
     return out, lse
+
+
+# ---- entry granularity ---------------------------------------------------------------------------------------------
+def janus_topk_entries(scores: torch.Tensor, n_entries: int, k: int, *, q_pos0: int, entry_size: int, want_count: bool = True,
+                       want_kth: bool = True):
+    """Top-k over entries of `entry_size` tokens: row t may select entries 0 .. (q_pos0 + t) // entry_size."""
+    lib = load()
+    M = scores.shape[0]
+    idx = torch.empty((M, k), dtype=torch.int32, device=scores.device)
+    count = torch.empty((M,), dtype=torch.int32, device=scores.device) if want_count else None
+    kth = torch.empty((M,), dtype=torch.float32, device=scores.device) if want_kth else None
+    rc = lib.janus_topk_entries(_ptr(scores), scores.stride(0), M, int(n_entries), int(q_pos0), int(entry_size), int(k), _ptr(idx),
+                                _ptr(count), _ptr(kth), _ptr(dev_status_tensor()), _stream())
+    _check(rc, "janus_topk_entries")
+    return idx, count, kth
+
+
+def janus_entry_expand(idx_entries: torch.Tensor, *, q_pos0: int, entry_size: int) -> torch.Tensor:
+    """Entry selection [M, k_e] -> token selection [M, k_e * entry_size] (tokens after the row's position become -1)."""
+    lib = load()
+    M, k_e = idx_entries.shape
+    out = torch.empty((M, k_e * entry_size), dtype=torch.int32, device=idx_entries.device)
+    rc = lib.janus_entry_expand(_ptr(idx_entries), M, k_e, int(entry_size), int(q_pos0), _ptr(out), _stream())
+    _check(rc, "janus_entry_expand")
+    return out
 
 
 # ---- decode step over a batch of sessions -------------------------------------------------------------------------

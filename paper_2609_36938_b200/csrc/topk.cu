@@ -31,6 +31,35 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_
     topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix64), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh);
 }
 
+// Entry granularity (footnote of Sec. 2.2): columns are entries of `entry_size` consecutive tokens; row t (position
+// q_pos0 + t) may select the entries that hold a token at or before its position: entries 0 .. (q_pos0 + t) / entry_size.
+template <int CAP>
+__global__ void __launch_bounds__(TK_THREADS)
+topk_entries_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_entries, int64_t q_pos0, int entry_size, int k,
+                    int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    using TopkShared = TopkSharedT<CAP>;
+    TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
+    const int t = blockIdx.x;
+    int64_t prefix = (q_pos0 + t) / entry_size + 1;
+    if (prefix > n_entries) prefix = n_entries;
+    topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh);
+}
+
+// Token selection of an entry selection: slot e * E + j of row t = entry * E + j if that token is at or before q_pos0 + t.
+__global__ void entry_expand_kernel(const int32_t* __restrict__ idx_e, int M, int k_e, int entry_size, int64_t q_pos0,
+                                    int32_t* __restrict__ idx_tok) {
+    const int64_t n = static_cast<int64_t>(M) * k_e * entry_size;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t slot = i / entry_size;            // (t, e)
+        const int j = static_cast<int>(i - slot * entry_size);
+        const int64_t t = slot / k_e;
+        const int32_t ent = __ldg(idx_e + slot);
+        const int64_t tok = static_cast<int64_t>(ent) * entry_size + j;
+        idx_tok[i] = (ent >= 0 && tok <= q_pos0 + t) ? static_cast<int32_t>(tok) : -1;
+    }
+}
+
 // Batch form (decode over many sessions): row b starts at scores[row_offsets[b]] and has row_lengths[b] elements (or runs
 // up to the next row's start when row_lengths is NULL), every element visible.
 template <int CAP>
@@ -49,6 +78,38 @@ topk_ragged_kernel(const float* __restrict__ scores, const int64_t* __restrict__
 }
 
 }  // namespace janus
+
+extern "C" int janus_topk_entries(const float* scores, int64_t scores_ld, int M, int64_t n_entries, int64_t q_pos0, int entry_size, int k,
+                                  int32_t* idx, int32_t* count, float* kth, int32_t* /*dev_status*/, void* stream_) {
+    using namespace janus;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (M < 0 || n_entries < 0 || k <= 0 || q_pos0 < 0 || entry_size <= 0 || scores_ld < n_entries) return JANUS_ERR_INVALID_ARG;
+    if (n_entries >= (int64_t(1) << 31) - 8) return JANUS_ERR_UNSUPPORTED;
+    if (M == 0) return JANUS_OK;
+    if (!idx) return JANUS_ERR_INVALID_ARG;
+    if (n_entries > 0 && (!scores || !aligned16(scores) || (scores_ld & 3) != 0)) return JANUS_ERR_INVALID_ARG;
+    const size_t smem = sizeof(TopkSharedT<TK_CAP>);
+    JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_entries_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    topk_entries_kernel<TK_CAP><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_entries, q_pos0, entry_size, k, idx, count, kth);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
+
+extern "C" int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_size, int64_t q_pos0, int32_t* idx_tokens,
+                                  void* stream_) {
+    using namespace janus;
+    if (M < 0 || k_e < 0 || entry_size <= 0 || q_pos0 < 0) return JANUS_ERR_INVALID_ARG;
+    const int64_t n = static_cast<int64_t>(M) * k_e * entry_size;
+    if (n == 0) return JANUS_OK;
+    if (!idx_entries || !idx_tokens) return JANUS_ERR_INVALID_ARG;
+    if (static_cast<int64_t>(k_e) * entry_size > 2147483647) return JANUS_ERR_UNSUPPORTED;
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    entry_expand_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream_)>>>(idx_entries, M, k_e, entry_size, q_pos0,
+                                                                                                       idx_tokens);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
 
 extern "C" int janus_topk_batch(const float* scores, const int64_t* row_offsets, const int64_t* row_lengths, int B, int k, int32_t* idx,
                                 int32_t* count, float* kth, int32_t* /*dev_status*/, void* stream_) {
