@@ -96,3 +96,38 @@ def test_binding_refuses_host_tensors_and_missing_library(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libjanus.so")
     with pytest.raises(binding.JanusError):
         binding.load()
+
+
+def test_batch_entry_and_static_entry_validation(lib):
+    """Host-side rejection for the entry points added after the four basic calls (nothing is launched on these paths)."""
+    INVALID, UNSUPPORTED, TOO_SMALL = 1, 2, 3
+    fake = ctypes.c_void_p(0x1000)
+    # decode batch: missing offsets, max_keys beyond the key array, head count the ragged tensor-core mode does not take
+    sb = lambda **kw: lib.janus_indexer_scores_batch(kw.get("q", fake), fake, 128, fake, None, 0, None, None, None, kw.get("B", 4), kw.get("H", 64),
+                                                      128, kw.get("off", fake), 4096, kw.get("max_keys", 1024), 0, kw.get("sc", fake), None, None)
+    assert sb(off=None) == INVALID
+    assert sb(max_keys=5000) == INVALID
+    assert sb(sc=None) == INVALID
+    assert sb(H=32) == UNSUPPORTED
+    assert sb(B=0) == 0
+    assert lib.janus_topk_batch(fake, fake, None, 4, 0, fake, None, None, None, None) == INVALID          # k = 0
+    assert lib.janus_topk_batch(fake, None, None, 4, 8, fake, None, None, None, None) == INVALID          # no offsets
+    assert lib.janus_topk_batch(fake, fake, None, 0, 8, fake, None, None, None, None) == 0                # empty batch
+    pdb = lambda **kw: lib.janus_page_demand_batch(fake, 4, 8, kw.get("lim", fake), kw.get("page", 64), fake, kw.get("off", fake), 64, None,
+                                                   kw.get("bitmap", fake), fake, fake, fake, fake, None, None, None, None, 64, None, None)
+    assert pdb(page=0) == INVALID
+    assert pdb(lim=None) == INVALID
+    assert pdb(off=None) == INVALID
+    assert pdb(bitmap=None) == INVALID
+    assert lib.janus_sparse_attn_decode(fake, 4, 128, 576, fake, fake, 64 * 576, 576, 576, 1, 512, fake, 64, 64, fake, None, 0.04, fake, None,
+                                        None, None) == INVALID                                              # no table offsets
+    # entry granularity
+    assert lib.janus_topk_entries(fake, 64, 4, 64, 0, 0, 8, fake, None, None, None, None) == INVALID       # entry_size = 0
+    assert lib.janus_topk_entries(fake, 32, 4, 64, 0, 16, 8, fake, None, None, None, None) == INVALID      # ld < n_entries
+    assert lib.janus_entry_expand(None, 4, 8, 16, 0, fake, None) == INVALID
+    assert lib.janus_entry_expand(fake, 0, 8, 16, 0, fake, None) == 0
+    # built-in scratch: the size check comes before the device is touched
+    assert lib.janus_indexer_topk_static(fake, 64 * 128, fake, 128, fake, fake, 0, fake, None, None, 4096, 64, 128, 135168, 131072, 1, 1, 2048,
+                                         fake, None, None, None, None) == TOO_SMALL
+    assert lib.janus_indexer_topk_static(fake, 64 * 128, fake, 128, fake, None, 0, None, None, None, 8, 64, 128, 4096, 0, 1, 0, 0,
+                                         fake, None, None, None, None) == INVALID                           # k = 0
