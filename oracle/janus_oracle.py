@@ -65,11 +65,26 @@ def decode_e4m3(codes) -> np.ndarray:
     return _E4M3[np.asarray(codes, dtype=np.uint8)]
 
 
+def decode_e2m1(packed) -> np.ndarray:
+    """FP4 E2M1 keys (Sec. 5.1: indexer keys of one model family are stored in FP4), two per byte, element 2i in the low
+    nibble of byte i -> float64 [..., 2 * bytes].  OCP E2M1: 1 sign, 2 exponent (bias 1), 1 mantissa bit; exponent 0 is
+    subnormal (0 or 0.5); no infinities or NaNs: the magnitudes are 0, 0.5, 1, 1.5, 2, 3, 4, 6."""
+    b = np.asarray(packed, dtype=np.uint8)
+    codes = np.stack([b & 0xF, b >> 4], axis=-1).reshape(*b.shape[:-1], b.shape[-1] * 2)
+    sign = np.where(codes & 0x8, -1.0, 1.0)
+    e = ((codes >> 1) & 0x3).astype(np.float64)
+    m = (codes & 0x1).astype(np.float64)
+    mag = np.where(e == 0, 0.5 * m, (1.0 + 0.5 * m) * 2.0 ** (e - 1.0))
+    return sign * mag
+
+
 def decode(x, dtype: str) -> np.ndarray:
     if dtype == "bf16":
         return decode_bf16(x)
     if dtype == "fp8":
         return decode_e4m3(x)
+    if dtype == "fp4":
+        return decode_e2m1(x)
     if dtype == "f64":
         return np.asarray(x, dtype=np.float64)
     raise ValueError(dtype)
@@ -93,8 +108,9 @@ def indexer_scores(q, k, w, *, dtype: str = "bf16", q_scale=None, k_scale=None,
     Bias (optional): either the rank-1 product row_bias[t]*col_bias[s], or
     ``recency=(amp, tau)`` evaluated directly as amp*exp(-(q_pos0+t-s)/tau).
     ``rows`` selects query rows (default all); returns float64 [len(rows), n_keys]."""
-    qd = decode(q, dtype)
-    kd = decode(k, dtype)
+    # dtype "fp8+fp4k": FP8 queries, FP4 (E2M1, packed two per byte) keys with the same per-key scale convention
+    qd = decode(q, "fp8" if dtype == "fp8+fp4k" else dtype)
+    kd = decode(k, "fp4" if dtype == "fp8+fp4k" else dtype)
     M, H, D = qd.shape
     n_keys = kd.shape[0]
     w = np.asarray(w, dtype=np.float64)

@@ -436,3 +436,26 @@ def test_entry_topk_hand_case_and_unit_entries():
     sel = O.entry_topk(np.array([[0.5, 2.0, 1.0, 9.0]]), 2, q_pos0=9, entry_size=4)
     assert sel.tolist() == [[1, 2]]
     assert O.entry_expand(sel, q_pos0=9, entry_size=4).tolist() == [[4, 5, 6, 7, 8, 9, -1, -1]]
+
+
+# ---- FP4 keys -----------------------------------------------------------------------------------------------------------
+def test_e2m1_decode_table_and_packing_order():
+    # the sixteen codes against the format's definition written out by hand
+    want = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0, -0.0, -0.5, -1.0, -1.5, -2.0, -3.0, -4.0, -6.0]
+    packed = np.array([[(2 * i) | ((2 * i + 1) << 4) for i in range(8)]], dtype=np.uint8)     # codes 0..15 in element order
+    got = O.decode_e2m1(packed)[0]
+    assert got.tolist() == want and np.signbit(got[8])
+    # every E2M1 value is an E4M3 value: FP4 keys and the same numbers stored as FP8 must score identically
+    rng = np.random.default_rng(4)
+    codes = rng.integers(0, 16, size=(50, 32)).astype(np.uint8)
+    packed = (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)
+    vals = O.decode_e2m1(packed)
+    import torch
+    k8 = torch.from_numpy(vals.astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(O.decode_e4m3(k8), vals)
+    q = rng.integers(0, 120, size=(3, 4, 32)).astype(np.uint8)
+    w = rng.uniform(0, 1, (3, 4)).astype(np.float32)
+    qs, ks = rng.uniform(0.5, 2, 4).astype(np.float32), rng.uniform(0.5, 2, 50).astype(np.float32)
+    a = O.indexer_scores(q, packed, w, dtype="fp8+fp4k", q_scale=qs, k_scale=ks, causal=False)
+    b = O.indexer_scores(q, k8, w, dtype="fp8", q_scale=qs, k_scale=ks, causal=False)
+    assert np.array_equal(a, b)
