@@ -168,8 +168,10 @@ def run_decode(args):
     n_keys = (L + 1 + 3) // 4 * 4
     key_off = torch.arange(nb + 1, dtype=torch.int64, device="cuda") * n_keys
     row_len = torch.full((nb,), L + 1, dtype=torch.int64, device="cuda")
-    k_idx = torch.randint(0, 256, (nb * n_keys, D), dtype=torch.uint8, device="cuda", generator=g)
-    k_idx = torch.where((k_idx & 0x7f) >= 0x7f, k_idx & 0xf7, k_idx)          # no NaN codes
+    fp4 = args.decode_fp4_keys
+    k_idx = torch.randint(0, 256, (nb * n_keys, D // 2 if fp4 else D), dtype=torch.uint8, device="cuda", generator=g)
+    if not fp4:
+        k_idx = torch.where((k_idx & 0x7f) >= 0x7f, k_idx & 0xf7, k_idx)      # no NaN codes
     q_idx = torch.randint(0, 120, (nb, H, D), dtype=torch.uint8, device="cuda", generator=g)
     w = torch.rand((nb, H), device="cuda", generator=g) / 8
     q_scale = torch.ones((nb, H), device="cuda") / 64
@@ -186,7 +188,7 @@ def run_decode(args):
 
     def step(marks=None):
         if marks: marks[0].record()
-        B.janus_indexer_scores_batch(q_idx, k_idx, w, key_off, n_keys, q_scale=q_scale, k_scale=k_scale, scores=scores)
+        B.janus_indexer_scores_batch(q_idx, k_idx, w, key_off, n_keys, q_scale=q_scale, k_scale=k_scale, scores=scores, keys_fp4=fp4)
         if marks: marks[1].record()
         idx, _, _ = B.janus_topk_batch(scores, key_off, k, row_lengths=row_len, want_count=False, want_kth=False)
         if marks: marks[2].record()
@@ -209,10 +211,10 @@ def run_decode(args):
     per = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks]).mean(axis=0)
     total_ms = float(np.mean([m[0].elapsed_time(m[4]) for m in marks]))
     peaks = load_peaks()
-    key_bytes = nb * (L + 1) * (D + 4 + 4)                    # key row + its scale read, score written
+    key_bytes = nb * (L + 1) * ((D // 2 if fp4 else D) + 4 + 4)   # key row + its scale read, score written
     line = {"metric": "decode_tokens_per_sec_per_sparse_layer", "value": nb / (total_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
             "steps": args.steps, "ms_per_step": total_ms, "data": "synthetic (device-generated)", "dtype": "fp8_e4m3+bf16",
-            "config": {"workload": f"decode step: {nb} sessions x {L} cached tokens, k={k}, FP8 64x128 indexer, latent attention, page {page}"},
+            "config": {"workload": f"decode step: {nb} sessions x {L} cached tokens, k={k}, {'FP8 queries / FP4 keys' if fp4 else 'FP8'} 64x128 indexer, latent attention, page {page}"},
             "kernels": {"indexer_scores_batch": {"ms": float(per[0]), "gbs": key_bytes / (per[0] * 1e-3) / 1e9,
                                                  "frac_hbm_peak": key_bytes / (per[0] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
                         "topk_batch": {"ms": float(per[1]), "gbs": nb * (L + 1) * 4 / (per[1] * 1e-3) / 1e9},
@@ -236,6 +238,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the side measurement of janus_indexer_topk")
     ap.add_argument("--decode-batch", type=int, default=0, help="side workload: time one decode step over this many sessions instead")
+    ap.add_argument("--decode-fp4-keys", action="store_true", help="with --decode-batch: indexer keys stored as FP4 E2M1")
     args = ap.parse_args()
     if args.decode_batch > 0:
         run_decode(args)

@@ -46,6 +46,8 @@ extern "C" {
 /* dtype of the indexer operands */
 #define JANUS_DTYPE_BF16 0
 #define JANUS_DTYPE_FP8_E4M3 1
+#define JANUS_DTYPE_FP8_Q_FP4_K 2   /* janus_indexer_scores_batch only: FP8 E4M3 queries, FP4 E2M1 keys (Sec. 5.1), two per
+                                       byte, element 2i in the low nibble of byte i; k_stride_tok counts elements */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int janus_version(void);
@@ -271,6 +273,8 @@ int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_siz
  *                              contiguous, w [B, H_I], q_scale [B, H_I] or [H_I]; max_keys = an upper bound of the
  *                              longest session (host value, sizes the launch); total_keys = rows of k_idx.
  *                              Tensor-core path only: H_I = 64 and 128- or 256-byte rows, else JANUS_ERR_UNSUPPORTED.
+ *                              dtype JANUS_DTYPE_FP8_Q_FP4_K: keys packed two per byte (D_I = 128, k_idx 32-byte aligned,
+ *                              k_stride_tok a multiple of 64 elements), scales as for FP8.
  * janus_topk_batch             idx[b, 0:k) = top-k of the row_lengths[b] scores starting at scores[row_offsets[b]] (positions inside
  *                              the session, -1 padded), count / kth as in janus_topk.  row_offsets [B + 1] and row_lengths
  *                              [B] are int64 device arrays; row_lengths may be NULL (rows then run up to the next offset);

@@ -328,17 +328,19 @@ def janus_entry_expand(idx_entries: torch.Tensor, *, q_pos0: int, entry_size: in
 def janus_indexer_scores_batch(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, key_offsets: torch.Tensor, max_keys: int, *,
                                q_scale: Optional[torch.Tensor] = None, k_scale: Optional[torch.Tensor] = None,
                                row_bias: Optional[torch.Tensor] = None, col_bias: Optional[torch.Tensor] = None,
-                               scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+                               scores: Optional[torch.Tensor] = None, keys_fp4: bool = False) -> torch.Tensor:
     """One query row per session against that session's keys.  q_idx [B,H,D]; k_idx [total_keys, D] (sessions concatenated);
-    key_offsets [B+1] int64 on the device.  Returns scores [total_keys] fp32 in the same row numbering as k_idx."""
+    key_offsets [B+1] int64 on the device.  Returns scores [total_keys] fp32 in the same row numbering as k_idx.
+    keys_fp4: k_idx is uint8 [total_keys, D/2], FP4 E2M1 packed two per byte (queries FP8)."""
     lib = load()
     B_, H, D = q_idx.shape
     total = k_idx.shape[0]
-    dtype = _idx_dtype_code(q_idx)
+    dtype = 2 if keys_fp4 else _idx_dtype_code(q_idx)
+    k_stride = k_idx.stride(0) * (2 if keys_fp4 else 1)
     if scores is None:
         scores = torch.empty((total,), dtype=torch.float32, device=q_idx.device)
     qs_stride = H if (q_scale is not None and q_scale.dim() == 2) else 0
-    rc = lib.janus_indexer_scores_batch(_ptr(q_idx), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
+    rc = lib.janus_indexer_scores_batch(_ptr(q_idx), _ptr(k_idx), k_stride, _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
                                         _ptr(row_bias), _ptr(col_bias), B_, H, D, _ptr(key_offsets), total, int(max_keys), dtype,
                                         _ptr(scores), _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_indexer_scores_batch")

@@ -56,6 +56,9 @@ struct TcCandParams {
     // ragged batch mode (decode over many sessions): query row b scores the keys key_offsets[b] .. key_offsets[b+1] of one
     // concatenated key array, no causal mask, and its scores go to scores[key_offsets[b] + s]
     const int64_t* key_offsets;
+    // ragged batch mode only: keys are FP4 E2M1, two per byte; the TMA expands 16 of them into the first 8 bytes of every
+    // 16-byte shared-memory chunk, which is the layout the f8f6f4 MMA expects for 4-bit operands
+    int k_fp4;
 };
 
 // Candidate mode stages appends in shared memory: each epilogue warp owns, for each of its (at most TC_CAND_TPW) tokens,
@@ -203,7 +206,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 const uint32_t ph = static_cast<uint32_t>(it / stages) & 1u;
                 if (!mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u) || *aborted) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); break; }
                 const uint32_t kf = smem_u32(&bars->k_full[s]);
-                mbar_expect_tx(kf, static_cast<uint32_t>(k_stage_bytes));
+                // packed 4-bit keys: the copy is counted in the bytes it reads (half of what it occupies in shared memory)
+                mbar_expect_tx(kf, static_cast<uint32_t>((RAGGED && cp.k_fp4) ? k_stage_bytes / 2 : k_stage_bytes));
                 for (int a = 0; a < atoms; ++a)
                     tma_load_2d(smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128), &tmap_k, a * atom_elems,
                                 static_cast<int>(key_base) + (tile_begin + it) * TC_KEYS, kf);
@@ -218,7 +222,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_vis > 0) {
-            constexpr uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N);   // ragged: only the first query row's heads
+            // ragged: only the first query row's heads (N = H); its keys (the A operand) may be E2M1 (format 5) against E4M3 queries
+            const uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N) | ((RAGGED && FP8 && cp.k_fp4) ? (5u << 7) : 0u);
             bool ok = mbar_wait(smem_u32(&bars->q_full), 0);
             uint32_t cnt = 0;
             for (int it = 0; it < n_vis && ok; ++it) {
@@ -381,7 +386,9 @@ bool make_tmap_2d_sw128(CUtensorMap* map, const void* base, int elem_bytes, uint
     const cuuint64_t strides[1] = {row_pitch_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    // elem_bytes 0: 4-bit elements, 16 of them expanded to a 16-byte aligned shared-memory chunk (box_cols must be 128)
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                   : elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B;
     return enc(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -421,7 +428,7 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
     p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = ld; p.n_keys = n_keys; p.q_pos0 = q_pos0;
     p.M = M; p.H = H; p.causal = causal; p.dev_status = dev_status;
-    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap, nullptr};
+    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap, nullptr, 0};
     p.atoms = D * esz / 128;
     p.nq = p.atoms == 1 ? 4 : 2;
     const int tps = TC_N / H;
@@ -476,6 +483,7 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
 // Ragged batch (decode): B query rows, row b against keys key_offsets[b] .. key_offsets[b+1] of one concatenated array.
 bool indexer_tc_batch_supported(int B, int H, int D, int64_t total_keys, int dtype) {
     const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
+    if (dtype == JANUS_DTYPE_FP8_Q_FP4_K && D != 128) return false;      // the packed 4-bit TMA box is 128 elements
     return H == 64 && (row_bytes == 128 || row_bytes == 256) && static_cast<int64_t>(B) * H < (int64_t(1) << 31) &&
            total_keys < (int64_t(1) << 31) - 256 && B <= 65535;
 }
@@ -484,13 +492,14 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
                             int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int B, int H, int D,
                             int64_t total_keys, int64_t max_keys, const int64_t* key_offsets, int dtype, float* scores, int32_t* dev_status,
                             cudaStream_t stream) {
-    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3;
+    const bool k_fp4 = dtype == JANUS_DTYPE_FP8_Q_FP4_K;
+    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3 || k_fp4;
     const int esz = fp8 ? 1 : 2;
     TcParams p;
     p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
     p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = 0; p.n_keys = total_keys; p.q_pos0 = 0;
     p.M = B; p.H = H; p.causal = 0; p.dev_status = dev_status;
-    const TcCandParams cp{nullptr, nullptr, nullptr, 0, key_offsets};
+    const TcCandParams cp{nullptr, nullptr, nullptr, 0, key_offsets, k_fp4 ? 1 : 0};
     p.atoms = D * esz / 128;
     p.nq = 1;
     const int tps = TC_N / H;
@@ -511,8 +520,12 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
     CUtensorMap tq, tk;
     const uint32_t box_cols = fp8 ? 128 : 64;
     if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(B) * H, D, static_cast<uint64_t>(D) * esz, TC_N, box_cols)) return JANUS_ERR_CUDA;
-    if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(total_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols))
+    if (k_fp4) {
+        if (!make_tmap_2d_sw128(&tk, k_idx, 0, static_cast<uint64_t>(total_keys), D, static_cast<uint64_t>(k_stride_tok) / 2, TC_KEYS, 128))
+            return JANUS_ERR_CUDA;
+    } else if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(total_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols)) {
         return JANUS_ERR_CUDA;
+    }
     return fp8 ? launch_tc<64, true, false, true>(tq, tk, p, cp, grid, smem, stream) : launch_tc<64, false, false, true>(tq, tk, p, cp, grid, smem, stream);
 }
 

@@ -94,8 +94,12 @@ extern "C" int janus_indexer_scores_batch(const void* q_idx, const void* k_idx, 
                                           int B, int H_I, int D_I, const int64_t* key_offsets, int64_t total_keys, int64_t max_keys,
                                           int dtype, float* scores, int32_t* dev_status, void* stream_) {
     using namespace janus;
+    // FP4 keys: the shared checks see an FP8 problem (queries are FP8, the scales are the same); the key array has its own rules
+    const bool k_fp4 = dtype == JANUS_DTYPE_FP8_Q_FP4_K;
+    if (k_fp4 && B > 0 && total_keys > 0 &&
+        (D_I != 128 || (k_stride_tok % 64) != 0 || (reinterpret_cast<uintptr_t>(k_idx) & 31u) != 0)) return k_idx ? JANUS_ERR_UNSUPPORTED : JANUS_ERR_INVALID_ARG;
     const int vrc = validate_indexer_args(q_idx, static_cast<int64_t>(H_I) * D_I, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale,
-                                          row_bias, col_bias, B, H_I, D_I, total_keys, 0, dtype);
+                                          row_bias, col_bias, B, H_I, D_I, total_keys, 0, k_fp4 ? JANUS_DTYPE_FP8_E4M3 : dtype);
     if (vrc != JANUS_OK) return vrc;
     if (max_keys < 0 || max_keys > total_keys) return JANUS_ERR_INVALID_ARG;
     if (B == 0 || total_keys == 0) return JANUS_OK;

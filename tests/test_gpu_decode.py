@@ -114,3 +114,30 @@ def test_decode_batch_matches_oracle_session_by_session(dtype):
     assert got["pages"] == sorted(all_pages)
     assert got["runs"] == [tuple(r) for r in O.maximal_runs(sorted(all_pages))]
     assert got["miss"] == sorted(all_pages)          # nothing declared resident
+
+
+def test_decode_indexer_with_fp4_keys():
+    # indexer keys stored as FP4 E2M1, two per byte (Sec. 5.1), FP8 queries: the same ragged batch call with another key format
+    lengths = [9000, 129, 20001, 40, 3333]
+    rng = np.random.default_rng(17)
+    nb, H, D = len(lengths), 64, 128
+    key_off = [0]
+    for L in lengths:
+        key_off.append(key_off[-1] + (L + 1 + 3) // 4 * 4)
+    total = key_off[-1]
+    codes = rng.integers(0, 16, size=(total, D)).astype(np.uint8)
+    packed = (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)          # element 2i in the low nibble of byte i
+    q = W.to_e4m3_bits(2 * rng.standard_normal((nb, H, D)).astype(np.float32))
+    w = (rng.uniform(0, 1, (nb, H)) / 8).astype(np.float32)
+    q_scale = np.exp2(rng.uniform(-2, 2, (nb, H))).astype(np.float32)
+    k_scale = np.exp2(rng.uniform(-1, 1, total)).astype(np.float32)
+    off = torch.tensor(key_off, dtype=torch.int64, device="cuda")
+    scores = B.janus_indexer_scores_batch(B.to_device(q, "fp8"), torch.from_numpy(packed).cuda(), B.to_device(w, "f32"), off, max(lengths) + 4,
+                                          q_scale=B.to_device(q_scale, "f32"), k_scale=B.to_device(k_scale, "f32"), keys_fp4=True)
+    B.check_dev_status()
+    got = scores.cpu().numpy()
+    for i, L in enumerate(lengths):
+        ks = slice(key_off[i], key_off[i] + L + 1)
+        ref = O.indexer_scores(q[i:i + 1], packed[ks], w[i:i + 1], dtype="fp8+fp4k", q_scale=q_scale[i:i + 1], k_scale=k_scale[ks],
+                               q_pos0=L, causal=True)
+        Hp.assert_scores_close(got[ks][None, :], ref, 1e-4, f"session {i} scores (fp4 keys)")
