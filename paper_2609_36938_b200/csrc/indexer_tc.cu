@@ -201,9 +201,9 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 for (int a = 0; a < atoms; ++a)
                     tma_load_2d(smem_u32(q_smem + j * q_sub_bytes + a * TC_N * 128), &tmap_q, a * atom_elems, (t0 + j * TPS) * H, qf);
             int issued = 0;
-            for (int it = 0; it < n_vis; ++it) {
-                const int s = it % stages;
-                const uint32_t ph = static_cast<uint32_t>(it / stages) & 1u;
+            int s = 0;                 // ring stage and its phase bit, advanced per tile (a division per tile costs a thread
+            uint32_t ph = 0;           // that issues everything on its own more than the copy it starts)
+            for (int it = 0; it < n_vis; ++it, s = (s + 1 == stages ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                 if (!mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u) || *aborted) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); break; }
                 const uint32_t kf = smem_u32(&bars->k_full[s]);
                 // packed 4-bit keys: the copy is counted in the bytes it reads (half of what it occupies in shared memory)
@@ -226,12 +226,16 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N) | ((RAGGED && FP8 && cp.k_fp4) ? (5u << 7) : 0u);
             bool ok = mbar_wait(smem_u32(&bars->q_full), 0);
             uint32_t cnt = 0;
-            for (int it = 0; it < n_vis && ok; ++it) {
-                const int s = it % stages;
-                const uint32_t ph = static_cast<uint32_t>(it / stages) & 1u;
+            // descriptors of the first key stage / first query sub-tile; every other operand is a constant number of 16-byte
+            // units further on, so stepping through the tiles is one 64-bit add
+            const uint64_t kdesc0 = umma_desc_sw128(smem_u32(k_smem)), qdesc0 = umma_desc_sw128(smem_u32(q_smem));
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < n_vis && ok; ++it, s = (s + 1 == stages ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                 ok = mbar_wait(smem_u32(&bars->k_full[s]), ph) && !*aborted;
                 if (!ok) break;
                 tc_fence_after();
+                const uint64_t kdesc_s = kdesc0 + static_cast<uint64_t>((s * k_stage_bytes) >> 4);
                 // ragged mode has one query sub-tile, so consecutive key tiles alternate between the two TMEM halves
                 for (int j = 0; j < nq; ++j, ++cnt) {
                     const uint32_t slot = cnt & 1u, use = cnt >> 1;
@@ -241,11 +245,11 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                     const uint32_t d_tmem = tmem_base + slot * TC_N;
                     uint32_t acc = 0;
                     for (int a = 0; a < atoms; ++a) {
-                        const uint32_t ka = smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128);
-                        const uint32_t qa = smem_u32(q_smem + j * q_sub_bytes + a * TC_N * 128);
+                        const uint64_t ka = kdesc_s + static_cast<uint64_t>((a * TC_KEYS * 128) >> 4);
+                        const uint64_t qa = qdesc0 + static_cast<uint64_t>((j * q_sub_bytes + a * TC_N * 128) >> 4);
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per instruction (16 bf16 or 32 e4m3)
-                            umma<FP8>(d_tmem, umma_desc_sw128(ka + ks * 32), umma_desc_sw128(qa + ks * 32), idesc, acc);
+                            umma<FP8>(d_tmem, ka + 2 * ks, qa + 2 * ks, idesc, acc);
                             acc = 1;
                         }
                     }
