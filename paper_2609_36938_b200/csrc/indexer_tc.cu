@@ -112,12 +112,17 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
 }
 
 template <int H, bool FP8, bool CAND, bool RAGGED>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, RAGGED ? 2 : 1)
 indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p, const TcCandParams cp) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int TPS = TC_N / H;                      // tokens per query sub-tile
     const int atoms = p.atoms, nq = p.nq, stages = p.stages;
-    const int q_sub_bytes = atoms * TC_N * 128;        // one query sub-tile
+    // ragged mode keeps only what one query row needs (H rows of Q, H accumulator columns per slot), so that two CTAs fit an SM
+    constexpr int QROWS = RAGGED ? H : TC_N;           // rows of a query sub-tile in shared memory
+    constexpr int SLOT_COLS = RAGGED ? H : TC_N;       // TMEM columns of one accumulator slot
+    constexpr int TMEM_COLS = RAGGED ? 2 * H : 512;
+    static_assert(TMEM_COLS >= 32 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM allocations are powers of two of at least 32 columns");
+    const int q_sub_bytes = atoms * QROWS * 128;       // one query sub-tile
     const int k_stage_bytes = atoms * TC_KEYS * 128;   // one key tile
     unsigned char* q_smem = smem;
     unsigned char* k_smem = smem + nq * q_sub_bytes;
@@ -168,7 +173,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         prefetch_tensormap(&tmap_k);
     }
     if (warp == 1 && n_vis > 0) {
-        tmem_alloc(smem_u32(&bars->tmem_base), 512);
+        tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
         tmem_relinquish();
     }
     // per-column weights (w * q_scale) and per-token bias factors of this CTA
@@ -199,7 +204,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             mbar_expect_tx(qf, static_cast<uint32_t>(nq * q_sub_bytes));
             for (int j = 0; j < nq; ++j)
                 for (int a = 0; a < atoms; ++a)
-                    tma_load_2d(smem_u32(q_smem + j * q_sub_bytes + a * TC_N * 128), &tmap_q, a * atom_elems, (t0 + j * TPS) * H, qf);
+                    tma_load_2d(smem_u32(q_smem + j * q_sub_bytes + a * QROWS * 128), &tmap_q, a * atom_elems, (t0 + j * TPS) * H, qf);
             int issued = 0;
             int s = 0;                 // ring stage and its phase bit, advanced per tile (a division per tile costs a thread
             uint32_t ph = 0;           // that issues everything on its own more than the copy it starts)
@@ -242,11 +247,11 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                     ok = mbar_wait(smem_u32(&bars->tmem_empty[slot]), (use & 1u) ^ 1u) && !*aborted;
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + slot * TC_N;
+                    const uint32_t d_tmem = tmem_base + slot * SLOT_COLS;
                     uint32_t acc = 0;
                     for (int a = 0; a < atoms; ++a) {
                         const uint64_t ka = kdesc_s + static_cast<uint64_t>((a * TC_KEYS * 128) >> 4);
-                        const uint64_t qa = qdesc0 + static_cast<uint64_t>((j * q_sub_bytes + a * TC_N * 128) >> 4);
+                        const uint64_t qa = qdesc0 + static_cast<uint64_t>((j * q_sub_bytes + a * QROWS * 128) >> 4);
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per instruction (16 bf16 or 32 e4m3)
                             umma<FP8>(d_tmem, ka + 2 * ks, qa + 2 * ks, idesc, acc);
@@ -292,7 +297,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars->tmem_full[e]), use & 1u) && !*aborted;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + e * TC_N;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + e * SLOT_COLS;
                 const int tsub0 = t0 + j * TPS;
                 float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 auto store = [&](int tt, float v) {
@@ -366,7 +371,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     __syncthreads();
     if (warp == 1 && n_vis > 0) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -507,10 +512,13 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
     p.atoms = D * esz / 128;
     p.nq = 1;
     const int tps = TC_N / H;
-    const int q_bytes = p.nq * p.atoms * TC_N * 128;
+    const int q_bytes = p.nq * p.atoms * H * 128;           // one query row: H (head) rows of the B operand
     const int k_stage = p.atoms * TC_KEYS * 128;
     const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + 2 * p.nq * tps) + static_cast<int>(sizeof(TcBarriers)) + 16;
-    p.stages = (TC_SMEM_BUDGET - q_bytes - tail) / k_stage;
+    // One query row per CTA leaves the single MMA-issuing thread as the limit of a CTA, so two CTAs share an SM: each gets
+    // half of the SM's shared memory (less the 1 KB the system keeps per CTA), half of TMEM and at most 96 registers a thread.
+    const int budget = (227 * 1024) / 2 - 1024;
+    p.stages = (budget - q_bytes - tail) / k_stage;
     if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
     if (p.stages < 2) return JANUS_ERR_UNSUPPORTED;
     const size_t smem = static_cast<size_t>(q_bytes) + static_cast<size_t>(p.stages) * k_stage + tail;
@@ -523,7 +531,7 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
     dim3 grid((max_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, B);
     CUtensorMap tq, tk;
     const uint32_t box_cols = fp8 ? 128 : 64;
-    if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(B) * H, D, static_cast<uint64_t>(D) * esz, TC_N, box_cols)) return JANUS_ERR_CUDA;
+    if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(B) * H, D, static_cast<uint64_t>(D) * esz, H, box_cols)) return JANUS_ERR_CUDA;
     if (k_fp4) {
         if (!make_tmap_2d_sw128(&tk, k_idx, 0, static_cast<uint64_t>(total_keys), D, static_cast<uint64_t>(k_stride_tok) / 2, TC_KEYS, 128))
             return JANUS_ERR_CUDA;
