@@ -46,8 +46,11 @@ extern "C" {
 /* dtype of the indexer operands */
 #define JANUS_DTYPE_BF16 0
 #define JANUS_DTYPE_FP8_E4M3 1
-#define JANUS_DTYPE_FP8_Q_FP4_K 2   /* janus_indexer_scores_batch only: FP8 E4M3 queries, FP4 E2M1 keys (Sec. 5.1), two per
-                                       byte, element 2i in the low nibble of byte i; k_stride_tok counts elements */
+#define JANUS_DTYPE_FP8_Q_FP4_K 2   /* FP8 E4M3 queries, FP4 E2M1 keys (Sec. 5.1), two per byte, element 2i in the low nibble of
+                                       byte i; k_stride_tok counts elements (a multiple of 64), k_idx is 32-byte aligned,
+                                       D_I = 128, scales as for FP8.  Taken by janus_indexer_scores, janus_indexer_topk(_static)
+                                       and janus_indexer_scores_batch, on tensor-core shapes only (else JANUS_ERR_UNSUPPORTED);
+                                       janus_indexer_topk then works through a score matrix in its workspace */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int janus_version(void);

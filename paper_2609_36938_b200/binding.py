@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG_DIR, "libjanus.so")
 JANUS_OK = 0
 ERR_NAMES = {1: "JANUS_ERR_INVALID_ARG", 2: "JANUS_ERR_UNSUPPORTED", 3: "JANUS_ERR_WORKSPACE_TOO_SMALL", 4: "JANUS_ERR_CUDA"}
 DEV_NAMES = {101: "JANUS_DEV_INDEX_OUT_OF_RANGE", 102: "JANUS_DEV_CAPACITY_EXCEEDED", 103: "JANUS_DEV_WAIT_TIMEOUT"}
-DTYPE_BF16, DTYPE_FP8_E4M3 = 0, 1
+DTYPE_BF16, DTYPE_FP8_E4M3, DTYPE_FP8_Q_FP4_K = 0, 1, 2
 
 # every symbol include/janus.h declares
 EXPORTS = [
@@ -149,25 +149,36 @@ def _idx_dtype_code(t: torch.Tensor) -> int:
     raise JanusError(f"indexer operands must be bfloat16 or E4M3 bytes, got {t.dtype}")
 
 
+def _idx_dtypes(q_idx: torch.Tensor, k_idx: torch.Tensor, keys_fp4: bool):
+    """(dtype code, key row stride in elements) of a query / key pair."""
+    dtype = _idx_dtype_code(q_idx)
+    if keys_fp4:
+        if dtype != DTYPE_FP8_E4M3 or k_idx.dtype != torch.uint8:
+            raise JanusError("FP4 keys are uint8 (two per byte) and go with E4M3 queries")
+        return DTYPE_FP8_Q_FP4_K, k_idx.stride(0) * 2
+    if _idx_dtype_code(k_idx) != dtype:
+        raise JanusError("q_idx and k_idx must share a dtype")
+    return dtype, k_idx.stride(0)
+
+
 def janus_indexer_scores(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, *, q_scale: Optional[torch.Tensor] = None,
                          k_scale: Optional[torch.Tensor] = None, row_bias: Optional[torch.Tensor] = None,
                          col_bias: Optional[torch.Tensor] = None, q_pos0: int = 0, causal: bool = True,
-                         scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+                         scores: Optional[torch.Tensor] = None, keys_fp4: bool = False) -> torch.Tensor:
     """scores[t,s] = sum_h w[t,h] relu(<q_idx[t,h], k_idx[s]>) (+ row_bias[t] col_bias[s]); -inf where masked.
-    q_idx [M,H,D], k_idx [n_keys,D] (bf16 or E4M3 bytes), w [M,H] fp32.  Returns [M, ld] fp32, ld >= n_keys."""
+    q_idx [M,H,D], k_idx [n_keys,D] (bf16 or E4M3 bytes), w [M,H] fp32.  Returns [M, ld] fp32, ld >= n_keys.
+    keys_fp4: k_idx is uint8 [n_keys, D/2], FP4 E2M1 packed two per byte (queries FP8)."""
     lib = load()
     M, H, D = q_idx.shape
     n_keys = k_idx.shape[0]
-    dtype = _idx_dtype_code(q_idx)
-    if _idx_dtype_code(k_idx) != dtype:
-        raise JanusError("q_idx and k_idx must share a dtype")
+    dtype, k_stride = _idx_dtypes(q_idx, k_idx, keys_fp4)
     if scores is None:
         ld = (n_keys + 31) // 32 * 32
         scores = torch.empty((M, ld), dtype=torch.float32, device=q_idx.device)
     qs_stride = 0
     if q_scale is not None and q_scale.dim() == 2:
         qs_stride = H
-    rc = lib.janus_indexer_scores(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride,
+    rc = lib.janus_indexer_scores(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_stride, _ptr(w), _ptr(q_scale), qs_stride,
                                   _ptr(k_scale), _ptr(row_bias), _ptr(col_bias), M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype,
                                   _ptr(scores), scores.stride(0), None, 0, _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_indexer_scores")
@@ -191,15 +202,16 @@ def janus_topk(scores: torch.Tensor, n_keys: int, k: int, *, q_pos0: int = 0, ca
 def janus_indexer_topk(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor, k: int, *, q_scale: Optional[torch.Tensor] = None,
                        k_scale: Optional[torch.Tensor] = None, row_bias: Optional[torch.Tensor] = None,
                        col_bias: Optional[torch.Tensor] = None, q_pos0: int = 0, causal: bool = True, want_count: bool = True,
-                       want_kth: bool = True, workspace: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None):
+                       want_kth: bool = True, workspace: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None,
+                       keys_fp4: bool = False):
     """Indexer scores and per-row top-k in one call, without the score matrix.  Returns (idx [M,k], count | None, kth | None).
-    `workspace` (uint8 CUDA tensor) is allocated if not given or too small; pass one to reuse it across calls; `idx` likewise."""
+    `workspace` (uint8 CUDA tensor) is allocated if not given or too small; pass one to reuse it across calls; `idx` likewise.
+    keys_fp4: k_idx is uint8 [n_keys, D/2], FP4 E2M1 packed two per byte (queries FP8); this format goes through a score
+    matrix inside the workspace."""
     lib = load()
     M, H, D = q_idx.shape
     n_keys = k_idx.shape[0]
-    dtype = _idx_dtype_code(q_idx)
-    if _idx_dtype_code(k_idx) != dtype:
-        raise JanusError("q_idx and k_idx must share a dtype")
+    dtype, k_stride = _idx_dtypes(q_idx, k_idx, keys_fp4)
     need = int(lib.janus_indexer_topk_workspace_size(M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype, int(k)))
     if workspace is None or workspace.numel() < need:
         workspace = torch.empty((max(need, 16),), dtype=torch.uint8, device=q_idx.device)
@@ -210,7 +222,7 @@ def janus_indexer_topk(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tensor
     count = torch.empty((M,), dtype=torch.int32, device=q_idx.device) if want_count else None
     kth = torch.empty((M,), dtype=torch.float32, device=q_idx.device) if want_kth else None
     qs_stride = H if (q_scale is not None and q_scale.dim() == 2) else 0
-    rc = lib.janus_indexer_topk(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_idx.stride(0), _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
+    rc = lib.janus_indexer_topk(_ptr(q_idx), q_idx.stride(0), _ptr(k_idx), k_stride, _ptr(w), _ptr(q_scale), qs_stride, _ptr(k_scale),
                                 _ptr(row_bias), _ptr(col_bias), M, H, D, n_keys, int(q_pos0), int(bool(causal)), dtype, int(k), _ptr(idx),
                                 _ptr(count), _ptr(kth), _ptr(workspace), workspace.numel(), _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_indexer_topk")

@@ -212,7 +212,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 if (!mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u) || *aborted) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); break; }
                 const uint32_t kf = smem_u32(&bars->k_full[s]);
                 // packed 4-bit keys: the copy is counted in the bytes it reads (half of what it occupies in shared memory)
-                mbar_expect_tx(kf, static_cast<uint32_t>((RAGGED && cp.k_fp4) ? k_stage_bytes / 2 : k_stage_bytes));
+                mbar_expect_tx(kf, static_cast<uint32_t>((FP8 && cp.k_fp4) ? k_stage_bytes / 2 : k_stage_bytes));
                 for (int a = 0; a < atoms; ++a)
                     tma_load_2d(smem_u32(k_smem + s * k_stage_bytes + a * TC_KEYS * 128), &tmap_k, a * atom_elems,
                                 static_cast<int>(key_base) + (tile_begin + it) * TC_KEYS, kf);
@@ -227,8 +227,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_vis > 0) {
-            // ragged: only the first query row's heads (N = H); its keys (the A operand) may be E2M1 (format 5) against E4M3 queries
-            const uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N) | ((RAGGED && FP8 && cp.k_fp4) ? (5u << 7) : 0u);
+            // ragged: only the first query row's heads (N = H); the keys (the A operand) may be E2M1 (format 5) against E4M3 queries
+            const uint32_t idesc = umma_idesc(FP8 ? 0u : 1u, TC_KEYS, RAGGED ? H : TC_N) | ((FP8 && cp.k_fp4) ? (5u << 7) : 0u);
             bool ok = mbar_wait(smem_u32(&bars->q_full), 0);
             uint32_t cnt = 0;
             // descriptors of the first key stage / first query sub-tile; every other operand is a constant number of 16-byte
@@ -406,6 +406,7 @@ bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_
     if (!(H == 4 || H == 8 || H == 16 || H == 32 || H == 64)) return false;
     const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
     if (row_bytes != 128 && row_bytes != 256) return false;
+    if (dtype == JANUS_DTYPE_FP8_Q_FP4_K && D != 128) return false;     // the packed 4-bit TMA box is 128 elements
     if (q_stride_tok != static_cast<int64_t>(H) * D) return false;
     if (static_cast<int64_t>(M) * H >= (int64_t(1) << 31) || n_keys >= (int64_t(1) << 31) - 256) return false;
     return true;
@@ -415,6 +416,7 @@ bool indexer_tc_supported(int M, int H, int D, int64_t n_keys, int64_t q_stride_
 bool indexer_tc_candidates_supported(int H, int D, int dtype) {
     const int row_bytes = D * (dtype == JANUS_DTYPE_BF16 ? 2 : 1);
     const int nq_max = row_bytes == 128 ? 4 : 2;
+    if (dtype == JANUS_DTYPE_FP8_Q_FP4_K) return false;                 // the sample gather and the exact fallback read 8- and 16-bit keys
     return (H == 32 || H == 64) && (nq_max / 2) * (TC_N / H) <= TC_CAND_TPW;
 }
 
@@ -431,13 +433,14 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
                       int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias, const float* col_bias, int M, int H,
                       int D, int64_t n_keys, int64_t q_pos0, int causal, int dtype, float* scores, int64_t ld, int32_t* dev_status,
                       cudaStream_t stream, const float* thr, int32_t* cand_cnt, void* cand, int cand_cap) {
-    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3;
+    const bool k_fp4 = dtype == JANUS_DTYPE_FP8_Q_FP4_K;
+    const bool fp8 = dtype == JANUS_DTYPE_FP8_E4M3 || k_fp4;
     const int esz = fp8 ? 1 : 2;
     TcParams p;
     p.w = w; p.q_scale = q_scale; p.q_scale_stride_tok = q_scale_stride_tok; p.k_scale = k_scale;
     p.row_bias = row_bias; p.col_bias = col_bias; p.scores = scores; p.ld = ld; p.n_keys = n_keys; p.q_pos0 = q_pos0;
     p.M = M; p.H = H; p.causal = causal; p.dev_status = dev_status;
-    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap, nullptr, 0};
+    const TcCandParams cp{thr, cand_cnt, static_cast<int2*>(cand), cand_cap, nullptr, k_fp4 ? 1 : 0};
     p.atoms = D * esz / 128;
     p.nq = p.atoms == 1 ? 4 : 2;
     const int tps = TC_N / H;
@@ -465,8 +468,12 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     CUtensorMap tq, tk;
     const uint32_t box_cols = fp8 ? 128 : 64;
     if (!make_tmap_2d_sw128(&tq, q_idx, esz, static_cast<uint64_t>(M) * H, D, static_cast<uint64_t>(D) * esz, TC_N, box_cols)) return JANUS_ERR_CUDA;
-    if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(n_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols))
+    if (k_fp4) {   // packed 4-bit keys: the copy expands 16 of them into the low halves of a 16-byte chunk
+        if (!make_tmap_2d_sw128(&tk, k_idx, 0, static_cast<uint64_t>(n_keys), D, static_cast<uint64_t>(k_stride_tok) / 2, TC_KEYS, 128))
+            return JANUS_ERR_CUDA;
+    } else if (!make_tmap_2d_sw128(&tk, k_idx, esz, static_cast<uint64_t>(n_keys), D, static_cast<uint64_t>(k_stride_tok) * esz, TC_KEYS, box_cols)) {
         return JANUS_ERR_CUDA;
+    }
 
 #define JANUS_TC_CASE(HH, CC)                                                         \
     case HH:                                                                          \

@@ -41,16 +41,22 @@ int validate_indexer_args(const void* q_idx, int64_t q_stride_tok, const void* k
                           const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
                           const float* col_bias, int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int dtype) {
     if (M < 0 || H_I <= 0 || D_I <= 0 || n_keys < 0 || q_pos0 < 0) return JANUS_ERR_INVALID_ARG;
-    if (dtype != JANUS_DTYPE_BF16 && dtype != JANUS_DTYPE_FP8_E4M3) return JANUS_ERR_UNSUPPORTED;
+    const bool k_fp4 = dtype == JANUS_DTYPE_FP8_Q_FP4_K;
+    if (dtype != JANUS_DTYPE_BF16 && dtype != JANUS_DTYPE_FP8_E4M3 && !k_fp4) return JANUS_ERR_UNSUPPORTED;
     if ((D_I % 16) != 0) return JANUS_ERR_UNSUPPORTED;
     if (M == 0 || n_keys == 0) return JANUS_OK;
     const int esz = dtype == JANUS_DTYPE_BF16 ? 2 : 1;
     if (!q_idx || !k_idx || !w) return JANUS_ERR_INVALID_ARG;
     if (!aligned16(q_idx) || !aligned16(k_idx)) return JANUS_ERR_INVALID_ARG;
     if (q_stride_tok < static_cast<int64_t>(H_I) * D_I || k_stride_tok < D_I) return JANUS_ERR_INVALID_ARG;
-    if ((q_stride_tok * esz) % 16 != 0 || (k_stride_tok * esz) % 16 != 0) return JANUS_ERR_INVALID_ARG;
+    if ((q_stride_tok * esz) % 16 != 0) return JANUS_ERR_INVALID_ARG;
+    if (k_fp4) {   // two key elements per byte: rows start on 32-byte boundaries (what the 4-bit tensor-map type asks for)
+        if ((k_stride_tok % 64) != 0 || (reinterpret_cast<uintptr_t>(k_idx) & 31u) != 0) return JANUS_ERR_INVALID_ARG;
+    } else if ((k_stride_tok * esz) % 16 != 0) {
+        return JANUS_ERR_INVALID_ARG;
+    }
     if ((row_bias == nullptr) != (col_bias == nullptr)) return JANUS_ERR_INVALID_ARG;
-    if (dtype == JANUS_DTYPE_FP8_E4M3) {
+    if (dtype != JANUS_DTYPE_BF16) {
         if (!q_scale || !k_scale) return JANUS_ERR_INVALID_ARG;
         if (q_scale_stride_tok != 0 && q_scale_stride_tok != H_I) return JANUS_ERR_INVALID_ARG;
     } else if (q_scale || k_scale) {
@@ -85,6 +91,7 @@ extern "C" int janus_indexer_scores(const void* q_idx, int64_t q_stride_tok, con
     if (!(force_general && force_general[0] == '1') && indexer_tc_supported(M, H_I, D_I, n_keys, q_stride_tok, k_stride_tok, dtype))
         return launch_indexer_tc(q_idx, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias, M, H_I, D_I,
                                  n_keys, q_pos0, causal, dtype, scores, scores_ld, dev_status, stream);
+    if (dtype == JANUS_DTYPE_FP8_Q_FP4_K) return JANUS_ERR_UNSUPPORTED;   // 4-bit keys: tensor-core shapes only
     return launch_indexer_generic(q_idx, q_stride_tok, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias,
                                   M, H_I, D_I, n_keys, q_pos0, causal, dtype, scores, scores_ld, stream);
 }

@@ -141,3 +141,38 @@ def test_decode_indexer_with_fp4_keys():
         ref = O.indexer_scores(q[i:i + 1], packed[ks], w[i:i + 1], dtype="fp8+fp4k", q_scale=q_scale[i:i + 1], k_scale=k_scale[ks],
                                q_pos0=L, causal=True)
         Hp.assert_scores_close(got[ks][None, :], ref, 1e-4, f"session {i} scores (fp4 keys)")
+
+
+def test_prefill_indexer_and_selection_with_fp4_keys():
+    # append prefill over a key cache stored as FP4 E2M1 (Sec. 5.1): scores against the oracle on sampled rows, and the
+    # one-call indexer + top-k (which takes this key format through a score matrix in its workspace)
+    M, L, H, D, k = 70, 20011, 64, 128, 256
+    rng = np.random.default_rng(23)
+    S = L + M
+    codes = rng.integers(0, 16, size=(S, D)).astype(np.uint8)
+    packed = (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)
+    q = W.to_e4m3_bits(2 * rng.standard_normal((M, H, D)).astype(np.float32))
+    w = (rng.uniform(0, 1, (M, H)) / 8).astype(np.float32)
+    q_scale = np.exp2(rng.uniform(-2, 2, (M, H))).astype(np.float32)
+    k_scale = np.exp2(rng.uniform(-1, 1, S)).astype(np.float32)
+    qd, kd, wd = B.to_device(q, "fp8"), torch.from_numpy(packed).cuda(), B.to_device(w, "f32")
+    args = dict(q_scale=B.to_device(q_scale, "f32"), k_scale=B.to_device(k_scale, "f32"), q_pos0=L, causal=True, keys_fp4=True)
+    scores = B.janus_indexer_scores(qd, kd, wd, **args)
+    idx, cnt, kth = B.janus_indexer_topk(qd, kd, wd, k, **args)
+    B.check_dev_status()
+    got, idx_h = scores.cpu().numpy(), idx.cpu().numpy()
+    assert np.array_equal(cnt.cpu().numpy(), np.full(M, k))
+    for t in W.sample_rows(M, 5):
+        t = int(t)
+        ref = O.indexer_scores(q[t:t + 1], packed, w[t:t + 1], dtype="fp8+fp4k", q_scale=q_scale[t:t + 1], k_scale=k_scale, q_pos0=L + t,
+                               causal=True)
+        Hp.assert_scores_close(got[t:t + 1, :L + t + 1], ref[:, :L + t + 1], 1e-4, f"row {t} scores (fp4 keys)")
+        assert np.all(np.isneginf(got[t, L + t + 1:S]))
+        ok, msg = O.topk_row_agrees(idx_h[t], ref[0], L + t + 1, k)
+        assert ok, f"row {t}: {msg}"
+    # a shape outside the tensor-core kernel has no 4-bit path
+    lib = B.load()
+    sc = torch.empty((3, 64), dtype=torch.float32, device="cuda")
+    rc = lib.janus_indexer_scores(qd.data_ptr(), 5 * D, kd.data_ptr(), D, wd.data_ptr(), args["q_scale"].data_ptr(), 5, args["k_scale"].data_ptr(),
+                                  None, None, 3, 5, D, 64, 0, 1, 2, sc.data_ptr(), 64, None, 0, None, None)
+    assert rc == 2                                            # JANUS_ERR_UNSUPPORTED
