@@ -11,6 +11,8 @@
 // If the sample misjudges the row (fewer than k candidates, or more than the buffer holds) the
 // same exact selection runs over the row in global memory instead; that path is slower, never
 // wrong.  Rows that fit the buffer skip the sampling step.
+#include <algorithm>
+
 #include "topk_select.cuh"
 
 namespace janus {
@@ -25,10 +27,15 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using TopkShared = TopkSharedT<CAP>;
     TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
-    const int t = blockIdx.x;
-    int64_t prefix64 = causal ? min(n_keys, q_pos0 + t + 1) : n_keys;
-    if (prefix64 < 0) prefix64 = 0;
-    topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix64), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh);
+    // resident CTAs walk the rows with stride gridDim.x, each asking for the head of its next row ahead of time
+    for (int t = blockIdx.x; t < M; t += gridDim.x) {
+        const int64_t prefix64 = causal ? min(n_keys, q_pos0 + t + 1) : n_keys;
+        const int t_next = t + gridDim.x;
+        const int64_t prefix_next = t_next < M ? (causal ? min(n_keys, q_pos0 + t_next + 1) : n_keys) : 0;
+        topk_row(scores + static_cast<int64_t>(t) * ld, static_cast<int>(prefix64), k, t, idx + static_cast<int64_t>(t) * k, count, kth, sh,
+                 t_next < M ? scores + static_cast<int64_t>(t_next) * ld : nullptr, static_cast<int>(prefix_next));
+        __syncthreads();   // the selection state in shared memory is reused by the next row
+    }
 }
 
 // Entry granularity (footnote of Sec. 2.2): columns are entries of `entry_size` consecutive tokens; row t (position
@@ -147,14 +154,21 @@ extern "C" int janus_topk(const float* scores, int64_t scores_ld, int M, int64_t
         const double e = 4096.0 * k / n_max, r = e + 4.0 * sqrt(e) + 8.0;
         small = n_max * (r + 5.0 * sqrt(r)) / 4096.0 <= TK_CAP_SMALL && k <= TK_CAP_SMALL / 2;
     }
+    int n_sm = 0, dev = 0, per_sm = 0;
+    JANUS_CUDA_CHECK(cudaGetDevice(&dev));
+    JANUS_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     if (small) {
         const size_t smem = sizeof(TopkSharedT<TK_CAP_SMALL>);
         JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel<TK_CAP_SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        topk_rows_kernel<TK_CAP_SMALL><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+        JANUS_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_rows_kernel<TK_CAP_SMALL>, TK_THREADS, smem));
+        const int grid = std::min(M, std::max(1, per_sm) * n_sm);
+        topk_rows_kernel<TK_CAP_SMALL><<<grid, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
     } else {
         const size_t smem = sizeof(TopkSharedT<TK_CAP>);
         JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_rows_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        topk_rows_kernel<TK_CAP><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
+        JANUS_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_rows_kernel<TK_CAP>, TK_THREADS, smem));
+        const int grid = std::min(M, std::max(1, per_sm) * n_sm);
+        topk_rows_kernel<TK_CAP><<<grid, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_keys, q_pos0, causal, k, idx, count, kth);
     }
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
