@@ -156,18 +156,98 @@ __device__ __forceinline__ void keep_candidates16(const float4 (&x)[4], int e0, 
 
 __device__ __forceinline__ void topk_prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// ---- the three phases of a row (n > k), callable separately so that several CTAs can share the streaming pass of one row
+
+// Streaming threshold of a row as an order-preserving key (0: keep everything): the sample value of a rank a few standard
+// deviations below where the row's k-th value is expected.  Thread i reads 8 consecutive floats at an evenly spread,
+// 32-byte aligned offset; the candidate buffer of `sh` is the scratch.  Every thread of the CTA calls it; the result is
+// uniform and depends on the row only.
+template <class Sh>
+__device__ uint32_t topk_sample_threshold(const float* __restrict__ row, int n, int k, Sh& sh) {
+    const int tid = threadIdx.x;
+    uint32_t thr = 0u;
+    if (n > Sh::kCap) {
+        const float4* row4 = reinterpret_cast<const float4*>(row);
+        const int n8 = n >> 3;                       // complete 8-float groups
+        const int g = static_cast<int>((static_cast<int64_t>(tid) * (n8 - 1)) / (TK_THREADS - 1));
+        const float4 a = __ldcg(row4 + 2 * g), b = __ldcg(row4 + 2 * g + 1);
+        uint32_t* skey = sh.cand_key;                // the candidate buffer is free at this point
+        skey[tid * 8 + 0] = float_to_key(a.x); skey[tid * 8 + 1] = float_to_key(a.y);
+        skey[tid * 8 + 2] = float_to_key(a.z); skey[tid * 8 + 3] = float_to_key(a.w);
+        skey[tid * 8 + 4] = float_to_key(b.x); skey[tid * 8 + 5] = float_to_key(b.y);
+        skey[tid * 8 + 6] = float_to_key(b.z); skey[tid * 8 + 7] = float_to_key(b.w);
+        __syncthreads();
+        const float expect = static_cast<float>(TK_SAMPLE) * static_cast<float>(k) / static_cast<float>(n);
+        const int r = static_cast<int>(expect + 4.0f * sqrtf(expect) + 8.0f);
+        if (r < TK_SAMPLE) {
+            int dummy;
+            SmemSource s{skey, nullptr, TK_SAMPLE};
+            thr = select_kth(s, r, sh, &dummy);
+        }
+        __syncthreads();
+    }
+    return thr;
+}
+
+// One streaming pass over the 16-byte groups [f4_begin, f4_end) of the row (and, with `tail`, the n % 4 elements after the
+// last whole group): elements at or above the threshold go to the candidate buffer of `dst`, which may be another CTA's
+// shared memory (a cluster-mapped reference).
+template <class Sh>
+__device__ void topk_stream(const float* __restrict__ row, int n, int f4_begin, int f4_end, bool tail, uint32_t thr, Sh& dst) {
+    const int tid = threadIdx.x;
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    const float thr_f = thr == 0u ? __int_as_float(0xff800000) : key_to_float(thr);
+    constexpr int UNROLL = 4;                     // 16-byte loads in flight per thread
+    int i = f4_begin + tid;
+    for (; i + (UNROLL - 1) * TK_THREADS < f4_end; i += UNROLL * TK_THREADS) {
+        float4 x[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) x[u] = __ldcs(row4 + i + u * TK_THREADS);
+        keep_candidates16(x, 4 * i, 4 * TK_THREADS, thr_f, dst);
+    }
+    for (; i < f4_end; i += TK_THREADS) {
+        const float4 x = __ldcs(row4 + i);
+        keep_if_candidate(x.x, 4 * i, thr_f, dst);
+        keep_if_candidate(x.y, 4 * i + 1, thr_f, dst);
+        keep_if_candidate(x.z, 4 * i + 2, thr_f, dst);
+        keep_if_candidate(x.w, 4 * i + 3, thr_f, dst);
+    }
+    const int n4 = n >> 2;
+    if (tail && tid < n - 4 * n4) keep_if_candidate(__ldcg(row + 4 * n4 + tid), 4 * n4 + tid, thr_f, dst);
+}
+
+// Exact selection over the candidates in `sh` (over the whole row in global memory when the sample misjudged it: fewer than
+// k candidates, or more than the buffer holds) and emission of the k indices, count and k-th value.
+template <class Sh>
+__device__ void topk_finish(const float* __restrict__ row, int n, int k, int t, int32_t* __restrict__ out, int32_t* __restrict__ count,
+                            float* __restrict__ kth, Sh& sh) {
+    const int n_cand = sh.n_cand;
+    uint32_t T;
+    int n_eq;
+    if (n_cand >= k && n_cand <= Sh::kCap) {
+        SmemSource s{sh.cand_key, sh.cand_idx, n_cand};
+        T = select_kth(s, k, sh, &n_eq);
+        emit_selection(s, T, n_eq, out, sh);
+    } else {
+        GlobalSource s{row, n};
+        T = select_kth(s, k, sh, &n_eq);
+        emit_selection(s, T, n_eq, out, sh);
+    }
+    if (threadIdx.x == 0) {
+        if (count) count[t] = n < k ? n : k;
+        if (kth) kth[t] = key_to_float(T);
+    }
+}
+
 // Top-k of one fp32 row of n elements (16-byte aligned) by the whole CTA (TK_THREADS threads): out[0..k) receives the
 // indices (-1 padded), count[t] / kth[t] the number selected and the smallest selected value (either may be NULL).
 // `next_row` (may be NULL): the row this CTA takes next.  The sample sectors of that row are requested into L2 once this
 // row's streaming pass is over, so the next sample does not start with a DRAM round trip.  (Requesting the head of the next
 // row as well, 96 to 512 KB, made the kernel slower: 0.49 -> 0.50 .. 0.58 ms at 4096 rows of 135168.)
-
 template <class Sh>
 __device__ void topk_row(const float* __restrict__ row, int n, int k, int t, int32_t* __restrict__ out, int32_t* __restrict__ count,
                          float* __restrict__ kth, Sh& sh, const float* __restrict__ next_row = nullptr, int next_n = 0) {
-    constexpr int TK_CAP = Sh::kCap;
     const int tid = threadIdx.x;
-    const int n_sel = n < k ? n : k;
 
     if (tid == 0) { sh.n_cand = 0; sh.out_pos = 0; sh.eq_taken = 0; }
     __syncthreads();
@@ -191,73 +271,15 @@ __device__ void topk_row(const float* __restrict__ row, int n, int k, int t, int
         return;
     }
 
-    uint32_t thr = 0u;  // keep everything
-    const float4* row4 = reinterpret_cast<const float4*>(row);
-    if (n > TK_CAP) {
-        // ---- sample: thread i reads 8 consecutive floats at an evenly spread, 32-byte aligned offset
-        const int n8 = n >> 3;                       // complete 8-float groups
-        const int g = static_cast<int>((static_cast<int64_t>(tid) * (n8 - 1)) / (TK_THREADS - 1));
-        const float4 a = __ldcg(row4 + 2 * g), b = __ldcg(row4 + 2 * g + 1);
-        uint32_t* skey = sh.cand_key;                // the candidate buffer is free at this point
-        skey[tid * 8 + 0] = float_to_key(a.x); skey[tid * 8 + 1] = float_to_key(a.y);
-        skey[tid * 8 + 2] = float_to_key(a.z); skey[tid * 8 + 3] = float_to_key(a.w);
-        skey[tid * 8 + 4] = float_to_key(b.x); skey[tid * 8 + 5] = float_to_key(b.y);
-        skey[tid * 8 + 6] = float_to_key(b.z); skey[tid * 8 + 7] = float_to_key(b.w);
-        __syncthreads();
-        // rank in the sample whose value sits a few standard deviations below the true k-th
-        const float expect = static_cast<float>(TK_SAMPLE) * static_cast<float>(k) / static_cast<float>(n);
-        int r = static_cast<int>(expect + 4.0f * sqrtf(expect) + 8.0f);
-        if (r < TK_SAMPLE) {
-            int dummy;
-            SmemSource s{skey, nullptr, TK_SAMPLE};
-            thr = select_kth(s, r, sh, &dummy);
-        }
-        __syncthreads();
-    }
-
-    // ---- one streaming pass: keep elements at or above the threshold (a few per cent of the row)
-    {
-        const float thr_f = thr == 0u ? __int_as_float(0xff800000) : key_to_float(thr);
-        const int n4 = n >> 2;
-        constexpr int UNROLL = 4;                     // 16-byte loads in flight per thread
-        int i = tid;
-        for (; i + (UNROLL - 1) * TK_THREADS < n4; i += UNROLL * TK_THREADS) {
-            float4 x[UNROLL];
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) x[u] = __ldcs(row4 + i + u * TK_THREADS);
-            keep_candidates16(x, 4 * i, 4 * TK_THREADS, thr_f, sh);
-        }
-        for (; i < n4; i += TK_THREADS) {
-            const float4 x = __ldcs(row4 + i);
-            keep_if_candidate(x.x, 4 * i, thr_f, sh);
-            keep_if_candidate(x.y, 4 * i + 1, thr_f, sh);
-            keep_if_candidate(x.z, 4 * i + 2, thr_f, sh);
-            keep_if_candidate(x.w, 4 * i + 3, thr_f, sh);
-        }
-        if (tid < n - 4 * n4) keep_if_candidate(__ldcg(row + 4 * n4 + tid), 4 * n4 + tid, thr_f, sh);   // ragged tail
-    }
+    const uint32_t thr = topk_sample_threshold(row, n, k, sh);
+    topk_stream(row, n, 0, n >> 2, true, thr, sh);
     if (next_row != nullptr && next_n > Sh::kCap) {
         const int n8 = next_n >> 3;
         const int g = static_cast<int>((static_cast<int64_t>(tid) * (n8 - 1)) / (TK_THREADS - 1));
         topk_prefetch_l2(next_row + 8 * g);                                   // the sample sector this thread will read
     }
     __syncthreads();
-    const int n_cand = sh.n_cand;
-    uint32_t T;
-    int n_eq;
-    if (n_cand >= k && n_cand <= TK_CAP) {
-        SmemSource s{sh.cand_key, sh.cand_idx, n_cand};
-        T = select_kth(s, k, sh, &n_eq);
-        emit_selection(s, T, n_eq, out, sh);
-    } else {
-        GlobalSource s{row, n};
-        T = select_kth(s, k, sh, &n_eq);
-        emit_selection(s, T, n_eq, out, sh);
-    }
-    if (tid == 0) {
-        if (count) count[t] = n_sel;
-        if (kth) kth[t] = key_to_float(T);
-    }
+    topk_finish(row, n, k, t, out, count, kth, sh);
 }
 
 }  // namespace janus
