@@ -10,6 +10,7 @@ namespace janus {
 constexpr int TK_THREADS = 512;
 constexpr int TK_BUCKETS = 2048;
 constexpr int TK_SAMPLE = 4096;     // 512 threads x 8 floats (one 32-byte sector each)
+constexpr int TK_DIRECT = 256;      // a bucket of at most this many keys is ranked directly instead of split further
 
 template <int CAP>
 struct TopkSharedT {
@@ -22,7 +23,8 @@ struct TopkSharedT {
     int out_pos;
     int eq_taken;
     uint32_t red_lo, red_hi;
-    int sel_bucket, sel_above;
+    int sel_bucket, sel_above, sel_count;
+    int n_small;
 };
 
 struct SmemSource {
@@ -89,7 +91,7 @@ __device__ uint32_t select_kth(const Src& src, int need, Sh& sh, int* n_eq_take)
         if (above < need && need <= above + mine) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (above < need && need <= above + c[j]) { sh.sel_bucket = TK_BUCKETS - 1 - (4 * tid + j); sh.sel_above = above; }
+                if (above < need && need <= above + c[j]) { sh.sel_bucket = TK_BUCKETS - 1 - (4 * tid + j); sh.sel_above = above; sh.sel_count = c[j]; }
                 above += c[j];
             }
         }
@@ -99,7 +101,35 @@ __device__ uint32_t select_kth(const Src& src, int need, Sh& sh, int* n_eq_take)
         const uint32_t new_lo = lo + (b << shift);
         if (b < (range >> shift)) hi = new_lo + ((1u << shift) - 1u);   // the top bucket keeps hi (and cannot overflow)
         lo = new_lo;
+        const int m = sh.sel_count;                                    // keys inside [lo, hi]
         __syncthreads();
+        if (lo < hi && m <= TK_DIRECT) {
+            // Few keys are left: instead of two more histogram passes (each a sweep over the source plus a block scan), copy
+            // them out (the histogram array is free) and let one thread per key count the keys above and equal to its own.
+            uint32_t* small = reinterpret_cast<uint32_t*>(sh.hist);
+            if (tid == 0) sh.n_small = 0;
+            __syncthreads();
+            for (int i = tid; i < n; i += TK_THREADS) {
+                const uint32_t key = src.key_at(i);
+                if (key >= lo && key <= hi) small[atomicAdd(&sh.n_small, 1)] = key;
+            }
+            __syncthreads();
+            for (int i = tid; i < m; i += TK_THREADS) {
+                const uint32_t mine = small[i];
+                int g = 0, e = 0;
+                for (int j = 0; j < m; ++j) {
+                    const uint32_t other = small[j];
+                    g += other > mine ? 1 : 0;
+                    e += other == mine ? 1 : 0;
+                }
+                if (g < need && need <= g + e) { sh.red_lo = mine; sh.sel_above = need - g; }   // equal keys write equal values
+            }
+            __syncthreads();
+            const uint32_t T = sh.red_lo;
+            *n_eq_take = sh.sel_above;
+            __syncthreads();
+            return T;
+        }
     }
     *n_eq_take = need;   // lo == hi: `need` of the elements equal to lo complete the selection
     return lo;
