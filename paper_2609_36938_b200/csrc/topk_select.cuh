@@ -105,7 +105,7 @@ __device__ uint32_t select_kth(const Src& src, int need, Sh& sh, int* n_eq_take)
         __syncthreads();
         if (lo < hi && m <= TK_DIRECT) {
             // Few keys are left: instead of two more histogram passes (each a sweep over the source plus a block scan), copy
-            // them out (the histogram array is free) and let one thread per key count the keys above and equal to its own.
+            // them out (the histogram array is free) and count, for every key, the keys above and equal to it.
             uint32_t* small = reinterpret_cast<uint32_t*>(sh.hist);
             if (tid == 0) sh.n_small = 0;
             __syncthreads();
@@ -114,15 +114,17 @@ __device__ uint32_t select_kth(const Src& src, int need, Sh& sh, int* n_eq_take)
                 if (key >= lo && key <= hi) small[atomicAdd(&sh.n_small, 1)] = key;
             }
             __syncthreads();
-            for (int i = tid; i < m; i += TK_THREADS) {
+            for (int i = tid >> 5; i < m; i += TK_THREADS / 32) {      // a warp per key, its lanes striding over the others
                 const uint32_t mine = small[i];
                 int g = 0, e = 0;
-                for (int j = 0; j < m; ++j) {
+                for (int j = tid & 31; j < m; j += 32) {
                     const uint32_t other = small[j];
                     g += other > mine ? 1 : 0;
                     e += other == mine ? 1 : 0;
                 }
-                if (g < need && need <= g + e) { sh.red_lo = mine; sh.sel_above = need - g; }   // equal keys write equal values
+                g = __reduce_add_sync(0xffffffffu, g);
+                e = __reduce_add_sync(0xffffffffu, e);
+                if ((tid & 31) == 0 && g < need && need <= g + e) { sh.red_lo = mine; sh.sel_above = need - g; }   // equal keys write equal values
             }
             __syncthreads();
             const uint32_t T = sh.red_lo;
