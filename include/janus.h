@@ -274,7 +274,8 @@ int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_siz
  * janus_indexer_scores_batch   scores[key_offsets[b] + s] = indexer score of session b's query against its key s
  *                              (no causal mask: the new token sees all of its session's keys).  q_idx [B, H_I, D_I]
  *                              contiguous, w [B, H_I], q_scale [B, H_I] or [H_I]; max_keys = an upper bound of the
- *                              longest session (host value, sizes the launch); total_keys = rows of k_idx.
+ *                              longest session (host value, sizes the launch; at most total_keys, else
+ *                              JANUS_ERR_INVALID_ARG); total_keys = rows of k_idx.
  *                              Tensor-core path only: H_I = 64 and 128- or 256-byte rows, else JANUS_ERR_UNSUPPORTED.
  *                              dtype JANUS_DTYPE_FP8_Q_FP4_K: keys packed two per byte (D_I = 128, k_idx 32-byte aligned,
  *                              k_stride_tok a multiple of 64 elements), scales as for FP8.
