@@ -27,7 +27,7 @@
 //                so it runs about two tiles ahead of the softmax; O += P.V (4 MMAs 128x256x16) needs P;
 //   warps 1-3    gather: warp g owns the ring slots s with s % 3 == g, resolves its 32 rows through the page table (one
 //                half-tile ahead) and copies this CTA's bytes with 16-byte cp.async into the 128-byte-swizzled K-major
-//                layout, 8 rows x 64 bytes per instruction;
+//                layout, 4 rows x 128 bytes per instruction;
 //   warps 4-7    exchange: as soon as a partial logit tile is complete they take it into registers, free the logit
 //                buffer and send it to the peer; after a token's last tile they load the next token's queries (prefetched
 //                into L2 one token earlier);
@@ -279,8 +279,8 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         // barrier is at most one phase ahead of it, which the parity wait relies on.
         const int g = warp - 1;
         const int total_half = n_my * n_half;                  // half-tiles of all tokens of this cluster, counted globally
-        const int g_sub = lane & 3, g_rr = lane >> 2;          // this lane copies piece g_sub of the 64-byte groups of rows 8q + g_rr
-        const uint32_t g_sw0 = static_cast<uint32_t>((g_sub ^ g_rr) << 4), g_sw1 = static_cast<uint32_t>(((4 + g_sub) ^ g_rr) << 4);
+        const int g_sub = lane & 7, g_rr = lane >> 3;          // this lane copies piece g_sub of the 128-byte groups of rows 4q + g_rr
+        const uint32_t g_sw0 = static_cast<uint32_t>((g_sub ^ g_rr) << 4), g_sw1 = static_cast<uint32_t>((g_sub ^ (4 + g_rr)) << 4);   // even / odd q
         const int64_t seg_off = 512 * static_cast<int64_t>(c); // first owned byte of a row
         bool ok = true;
         LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
@@ -333,23 +333,22 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (!ok) break;
             if (lane == 0) sh->vmask[2 * buf + hf] = valid_mask;
             const uint32_t stage_base = smem_u32(k_smem + buf * LP_TILE_BYTES + hf * LP_HALF * 128);
-            // One instruction copies 64 contiguous bytes (4 lanes x 16) of each of 8 rows, so a row pointer is fetched from
-            // its owner lane once per 8 rows and every copy is a single instruction with immediate offsets: chunk ch of the
-            // owned bytes goes to atom ch/8, position (ch%8) ^ (r%8) inside the 128-byte row r.
+            // One instruction copies 128 contiguous bytes (8 lanes x 16, one whole line) of each of 4 rows, so a row pointer is
+            // fetched from its owner lane once per 4 rows and every copy is a single instruction with immediate offsets: the
+            // 128-byte group a of the owned bytes is row r of atom a, its 16-byte pieces at positions piece ^ (r % 8).
+            // (Half lines of 8 rows per instruction, the same number of instructions, were 2.4 % slower: the copies are
+            // bound by the rate at which the load/store unit takes these instructions, about 28 cycles each.)
             const uint32_t lo = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr)), hi32 = static_cast<uint32_t>(reinterpret_cast<uint64_t>(row_ptr) >> 32);
 #pragma unroll
-            for (int q = 0; q < LP_HALF / 8; ++q) {
-                const int r = 8 * q + g_rr;
+            for (int q = 0; q < LP_HALF / 4; ++q) {
+                const int r = 4 * q + g_rr;
                 const uint64_t pr = (static_cast<uint64_t>(__shfl_sync(0xffffffffu, hi32, r)) << 32) | __shfl_sync(0xffffffffu, lo, r);
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(pr) + g_sub * 16;
                 const uint32_t bytes = ((valid_mask >> r) & 1u) ? 16u : 0u;
-                const uint32_t d = stage_base + static_cast<uint32_t>(r * 128);
+                const uint32_t d = stage_base + static_cast<uint32_t>(r * 128) + ((q & 1) ? g_sw1 : g_sw0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) cp_async16(d + (i >> 1) * LP_K_ATOM_BYTES + ((i & 1) ? g_sw1 : g_sw0), src + i * 64, bytes);
-                if (c == 1u) {
-                    cp_async16(d + 4 * LP_K_ATOM_BYTES + g_sw0, src + 512, bytes);
-                    cp_async16(d + 4 * LP_K_ATOM_BYTES + g_sw1, src + 576, bytes);
-                }
+                for (int a = 0; a < 4; ++a) cp_async16(d + a * LP_K_ATOM_BYTES, src + a * 128, bytes);
+                if (c == 1u) cp_async16(d + 4 * LP_K_ATOM_BYTES, src + 512, bytes);
             }
             cp_async_commit();
             row_nxt = resolve(raw_nxt, tbl_nxt, tbl_n_nxt, valid_nxt);   // page-table load overlaps the copies in flight
