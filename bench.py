@@ -140,13 +140,26 @@ def run_reference(args, shp, sess):
         O.sparse_attention(sess["Q"], sess["k_pool"], sess["v_pool"], sess["page_table"], idx, page_size=shp.page_size,
                            softmax_scale=shp.softmax_scale, d_qk=shp.d_qk, d_v=shp.d_v, rows=rows)
 
+    # The oracle's matrix products run in the BLAS numpy links; a launcher that exports OMP_NUM_THREADS=1 (torchrun does)
+    # would pin it to one thread, so the thread count is set here to the cores this process may use, and reported.
+    cores = len(os.sched_getaffinity(0))
+    try:
+        from threadpoolctl import threadpool_info, threadpool_limits
+        limiter = threadpool_limits(limits=cores)
+    except Exception:
+        limiter, threadpool_info = None, None
     for _ in range(args.warmup_ref):
         step()
     t0 = time.perf_counter()
     for _ in range(args.steps_ref):
         step()
     dt = (time.perf_counter() - t0) / args.steps_ref
-    cores = len(os.sched_getaffinity(0))
+    if threadpool_info is not None:
+        used = [int(p.get("num_threads", 0)) for p in threadpool_info() if p.get("user_api") in ("blas", "openmp")]
+        if used:
+            cores = max(used)
+    if limiter is not None:
+        limiter.restore_original_limits()
     value = len(rows) / dt
     return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{len(rows)} of {shp.M} query rows (first, last, evenly spread), all {shp.S} keys, k={shp.k}; "
