@@ -1,13 +1,15 @@
 // janus_topk: per-row selection of the k largest scores over the causal prefix (Eq. 1, Sec. 2.2).
 //
-// One CTA per query row.  The row (0.5-1 MB of fp32 at 128K-256K keys) is read from HBM once:
+// A CTA works on one query row at a time; the CTAs resident on the device walk the rows with stride gridDim.x.  The row
+// (0.5-1 MB of fp32 at 128K-256K keys) is read from HBM once:
 //   1. a strided sample of the row (512 x 32-byte sectors) gives a conservative threshold whose
 //      expected rank is a little above k;
 //   2. one streaming pass with 16-byte loads keeps only the elements at or above that threshold
 //      in a shared-memory candidate buffer (~1.5-3 % of the row pass the one-compare filter);
-//   3. an exact selection runs on the candidates in shared memory: repeated 2048-bucket
-//      histograms over a shrinking key range (buckets are linear in the order-preserving integer
-//      key, so they spread over whatever range the scores occupy), until the k-th key is isolated.
+//   3. an exact selection runs on the candidates in shared memory: 2048-bucket histograms over a
+//      shrinking key range (buckets are linear in the order-preserving integer key, so they spread
+//      over whatever range the scores occupy) until the bucket of the k-th key holds at most 256
+//      keys, which are then ranked directly.
 // If the sample misjudges the row (fewer than k candidates, or more than the buffer holds) the
 // same exact selection runs over the row in global memory instead; that path is slower, never
 // wrong.  Rows that fit the buffer skip the sampling step.
