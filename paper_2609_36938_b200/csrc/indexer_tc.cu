@@ -23,6 +23,7 @@ using namespace ptx;
 constexpr int TC_KEYS = 128;        // keys per tile = MMA M
 constexpr int TC_N = 256;           // (token, head) rows per MMA = MMA N
 constexpr int TC_THREADS = 320;     // 1 TMA warp + 1 MMA warp + 8 epilogue warps
+constexpr int TC_THREADS_RAGGED = 192;   // ragged mode: one epilogue group (4 warps), so that four CTAs fit an SM
 constexpr int TC_SMEM_BUDGET = 227 * 1024;
 constexpr int TC_MAX_STAGES = 6;
 
@@ -112,7 +113,7 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
 }
 
 template <int H, bool FP8, bool CAND, bool RAGGED>
-__global__ void __launch_bounds__(TC_THREADS, RAGGED ? 2 : 1)
+__global__ void __launch_bounds__(RAGGED ? TC_THREADS_RAGGED : TC_THREADS, RAGGED ? 4 : 1)
 indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p, const TcCandParams cp) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int TPS = TC_N / H;                      // tokens per query sub-tile
@@ -177,7 +178,8 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         tmem_relinquish();
     }
     // per-column weights (w * q_scale) and per-token bias factors of this CTA
-    for (int n = threadIdx.x; n < nq * TC_N; n += TC_THREADS) {
+    constexpr int NTHREADS = RAGGED ? TC_THREADS_RAGGED : TC_THREADS;
+    for (int n = threadIdx.x; n < nq * TC_N; n += NTHREADS) {
         const int t = t0 + n / H, h = n % H;
         float v = 0.f;
         if (t < p.M) {
@@ -186,7 +188,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
         ws[n] = 0.5f * v;      // the epilogue forms 2 * relu
     }
-    for (int n = threadIdx.x; n < tpc; n += TC_THREADS) {
+    for (int n = threadIdx.x; n < tpc; n += NTHREADS) {
         rbs[n] = (p.row_bias != nullptr && t0 + n < p.M) ? p.row_bias[t0 + n] : 0.f;
         if constexpr (CAND) thrs[n] = t0 + n < p.M ? cp.thr[t0 + n] : 0.f;
     }
@@ -291,13 +293,14 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const float kscale = (FP8 && key_ok) ? p.k_scale[s] : 1.f;
             const float cb = (p.col_bias != nullptr && key_ok) ? p.col_bias[s] : 0.f;
             // score-matrix and candidate modes: group e drains the sub-tiles j = e, e+2, .. of every key tile (nq is even);
-            // ragged mode (nq = 1): group e drains the key tiles it = e, e+2, ..
-            for (int j = RAGGED ? ((it & 1) == e ? 0 : nq) : e; j < nq; j += 2) {
+            // ragged mode (nq = 1, one group): key tile `it` sits in slot it % 2
+            for (int j = RAGGED ? 0 : e; j < nq; j += 2) {
+                const int slot = RAGGED ? (it & 1) : e;     // ragged: the one group takes both slots in turn
                 const uint32_t use = static_cast<uint32_t>(it * nq + j) >> 1;
-                ok = mbar_wait(smem_u32(&bars->tmem_full[e]), use & 1u) && !*aborted;
+                ok = mbar_wait(smem_u32(&bars->tmem_full[slot]), use & 1u) && !*aborted;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + e * SLOT_COLS;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + slot * SLOT_COLS;
                 const int tsub0 = t0 + j * TPS;
                 float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 auto store = [&](int tt, float v) {
@@ -347,7 +350,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                         // every column of this TMEM half is in registers: hand it back before the last reduction
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[e]));
+                        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[slot]));
                     }
                     reduce_chunk<H>(rb, ws + j * TC_N + (c + 1) * 32, (c + 1) * 32, acc, store);
                 }
@@ -424,7 +427,7 @@ template <int H, bool FP8, bool CAND, bool RAGGED = false>
 static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, const TcCandParams& cp, dim3 grid, size_t smem,
                      cudaStream_t stream) {
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8, CAND, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    indexer_tc_kernel<H, FP8, CAND, RAGGED><<<grid, TC_THREADS, smem, stream>>>(tq, tk, p, cp);
+    indexer_tc_kernel<H, FP8, CAND, RAGGED><<<grid, RAGGED ? TC_THREADS_RAGGED : TC_THREADS, smem, stream>>>(tq, tk, p, cp);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
@@ -522,9 +525,10 @@ int launch_indexer_tc_batch(const void* q_idx, const void* k_idx, int64_t k_stri
     const int q_bytes = p.nq * p.atoms * H * 128;           // one query row: H (head) rows of the B operand
     const int k_stage = p.atoms * TC_KEYS * 128;
     const int tail = static_cast<int>(sizeof(float)) * (p.nq * TC_N + 2 * p.nq * tps) + static_cast<int>(sizeof(TcBarriers)) + 16;
-    // One query row per CTA leaves the single MMA-issuing thread as the limit of a CTA, so two CTAs share an SM: each gets
-    // half of the SM's shared memory (less the 1 KB the system keeps per CTA), half of TMEM and at most 96 registers a thread.
-    const int budget = (227 * 1024) / 2 - 1024;
+    // One query row per CTA leaves the single MMA-issuing thread as the limit of a CTA, so several CTAs share an SM: four with
+    // one-byte operands (each a quarter of the SM's shared memory less the 1 KB the system keeps per CTA, 2 x H of the 512
+    // TMEM columns, 6 warps of at most 80 registers), two with bf16 (a key stage is 32 KB).
+    const int budget = (227 * 1024) / (fp8 ? 4 : 2) - 1024;
     p.stages = (budget - q_bytes - tail) / k_stage;
     if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
     if (p.stages < 2) return JANUS_ERR_UNSUPPORTED;
