@@ -77,4 +77,43 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
     return warp_sums[warp] + incl - v;
 }
 
+// The same for three ints per thread at once (one set of barriers instead of three).  `warp_sums` holds 3 x 33 ints.
+template <int THREADS>
+__device__ __forceinline__ void block_exclusive_scan3(int (&v)[3], int* warp_sums, int (&excl)[3], int (&total)[3]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl[3] = {v[0], v[1], v[2]};
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int y = __shfl_up_sync(0xffffffffu, incl[q], d);
+            if (lane >= d) incl[q] += y;
+        }
+    }
+    __syncthreads();  // protect warp_sums from a previous use
+    if (lane == 31) {
+#pragma unroll
+        for (int q = 0; q < 3; ++q) warp_sums[33 * q + warp] = incl[q];
+    }
+    __syncthreads();
+    if (warp < 3) {   // warp q scans the warp totals of value q
+        const int q = warp;
+        const int sv = (lane < THREADS / 32) ? warp_sums[33 * q + lane] : 0;
+        int si = sv;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, si, d);
+            if (lane >= d) si += y;
+        }
+        if (lane < THREADS / 32) warp_sums[33 * q + lane] = si - sv;
+        if (lane == 31) warp_sums[33 * q + 32] = si;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        total[q] = warp_sums[33 * q + 32];
+        excl[q] = warp_sums[33 * q + warp] + incl[q] - v[q];
+    }
+}
+
 }  // namespace janus

@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(LIST_THREADS)
 page_lists_chunk_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ predicted, int n_words, int64_t n_phys_pages,
                         int32_t* pages, int32_t* n_pages, int32_t* runs, int32_t* n_runs, int32_t* miss_pages, int32_t* n_miss,
                         int32_t* miss_runs, int32_t* n_miss_runs, int64_t capacity, int32_t* dev_status) {
-    __shared__ int scan_scratch[40];
+    __shared__ int scan_scratch[3 * 33];
     const bool miss = blockIdx.y == 1;
     const uint32_t* a = bitmap;
     const uint32_t* not_b = miss ? predicted : nullptr;
@@ -172,19 +172,18 @@ page_lists_chunk_kernel(const uint32_t* __restrict__ bitmap, const uint32_t* __r
         c_st += __popc(starts_of(i, v));
         c_en += __popc(ends_of(i, v));
     }
-    int id_base, run_base, end_base, dummy;
-    dummy = block_exclusive_scan<LIST_THREADS>(c_id, scan_scratch, &id_base);
-    dummy = block_exclusive_scan<LIST_THREADS>(c_st, scan_scratch, &run_base);
-    dummy = block_exclusive_scan<LIST_THREADS>(c_en, scan_scratch, &end_base);
-    (void)dummy;
+    // ids, run starts and run ends are scanned together: one set of block barriers per scan instead of three
+    int before[3] = {c_id, c_st, c_en}, skip[3], bases[3];
+    block_exclusive_scan3<LIST_THREADS>(before, scan_scratch, skip, bases);
+    const int id_base = bases[0], run_base = bases[1], end_base = bases[2];
     // ---- this chunk
     const int i = base + threadIdx.x;
     const uint32_t v = word_at(i);
     const uint32_t starts = starts_of(i, v), ends = ends_of(i, v);
-    int tot_ids, tot_starts, tot_ends;
-    int o_id = block_exclusive_scan<LIST_THREADS>(__popc(v), scan_scratch, &tot_ids) + id_base;
-    int o_st = block_exclusive_scan<LIST_THREADS>(__popc(starts), scan_scratch, &tot_starts) + run_base;
-    int o_en = block_exclusive_scan<LIST_THREADS>(__popc(ends), scan_scratch, &tot_ends) + end_base;
+    int mine[3] = {__popc(v), __popc(starts), __popc(ends)}, offs[3], tots[3];
+    block_exclusive_scan3<LIST_THREADS>(mine, scan_scratch, offs, tots);
+    const int tot_ids = tots[0], tot_starts = tots[1];
+    int o_id = offs[0] + id_base, o_st = offs[1] + run_base, o_en = offs[2] + end_base;
     uint32_t m = v;
     while (m) {
         const int b = __ffs(m) - 1;
