@@ -110,6 +110,47 @@ def test_indexer_fp8_unit_scales_equals_bf16_on_representable_values():
     assert np.array_equal(a, b)
 
 
+def test_indexer_per_token_query_scales_hand_case_and_broadcast_axis():
+    # FP8 queries with one scale per (token, head) (Sec. 5.1 storage; Eq. 1 scoring): the scale multiplies head h of token t.
+    # Hand case, 2 tokens x 2 heads x 2 dims, 2 keys, every value exact in E4M3:
+    q = np.array([[[1, 2], [2, -1]],
+                  [[1, 2], [2, -1]]], dtype=np.float32)          # both tokens store the same codes: only the scales differ
+    k = np.array([[1, 1], [1, -1]], dtype=np.float32)
+    w = np.array([[1.0, 1.0], [1.0, 1.0]], dtype=np.float32)
+    qs = np.array([[1.0, 2.0], [4.0, 0.5]])                      # qs[t, h]
+    # code dots: h0: [3, -1]; h1: [1, 3]
+    # t=0: scales (1, 2): relu([3,-1]) + relu([2, 6]) = [5, 6];  t=1: scales (4, 0.5): relu([12,-4]) + relu([0.5,1.5]) = [12.5, 1.5]
+    sc = O.indexer_scores(W.to_e4m3_bits(q), W.to_e4m3_bits(k), w, dtype="fp8", q_scale=qs, k_scale=np.ones(2), causal=False)
+    assert np.array_equal(sc, np.array([[5.0, 6.0], [12.5, 1.5]]))
+    # a swapped broadcast axis would read qs[h, t]: (1, 4) for t=0 -> [3+4, 12] and fails the line above; check it is different
+    assert not np.array_equal(sc, np.array([[7.0, 12.0], [6.5, 1.5]]))
+    # a per-head vector repeated for every token is bit-identical to the 1-D call (non-square shape: a transposed use cannot broadcast)
+    rng = np.random.default_rng(14)
+    M, H, D, n = 5, 3, 8, 7
+    cq = W.to_e4m3_bits(rng.standard_normal((M, H, D)))
+    ck = W.to_e4m3_bits(rng.standard_normal((n, D)))
+    wv = rng.uniform(-1, 1, (M, H)).astype(np.float32)
+    per_head = (2.0 ** rng.uniform(-2, 2, H)).astype(np.float32)
+    ks = (2.0 ** rng.uniform(-4, 4, n)).astype(np.float32)
+    one_d = O.indexer_scores(cq, ck, wv, dtype="fp8", q_scale=per_head, k_scale=ks, q_pos0=2, causal=True)
+    two_d = O.indexer_scores(cq, ck, wv, dtype="fp8", q_scale=np.tile(per_head, (M, 1)), k_scale=ks, q_pos0=2, causal=True)
+    assert np.array_equal(one_d, two_d)
+    # scaling one token's scale row by c > 0 scales exactly that token's score row (ReLU is positively homogeneous)
+    qs2 = np.tile(per_head, (M, 1)).astype(np.float64)
+    qs2[3] *= 4.0
+    scaled = O.indexer_scores(cq, ck, wv, dtype="fp8", q_scale=qs2, k_scale=ks, causal=False)
+    base = O.indexer_scores(cq, ck, wv, dtype="fp8", q_scale=per_head, k_scale=ks, causal=False)
+    factor = np.ones((M, 1)); factor[3] = 4.0
+    np.testing.assert_allclose(scaled, base * factor, rtol=1e-13, atol=0)
+    # a scale on one head of one token equals that head's weight scaled instead (the scale sits outside the ReLU)
+    qs3 = np.tile(per_head, (M, 1)).astype(np.float64)
+    qs3[1, 2] *= 8.0
+    w3 = wv.astype(np.float64).copy()
+    w3[1, 2] *= 8.0
+    np.testing.assert_allclose(O.indexer_scores(cq, ck, wv, dtype="fp8", q_scale=qs3, k_scale=ks, causal=False),
+                               O.indexer_scores(cq, ck, w3, dtype="fp8", q_scale=per_head, k_scale=ks, causal=False), rtol=1e-13, atol=1e-300)
+
+
 def test_indexer_mask_counts_and_self_inclusion():
     rng = np.random.default_rng(4)
     L, M = 5, 4
