@@ -11,7 +11,10 @@
 // 128-key tiles past them through a TMA ring; each key tile feeds NQ MMAs (128 x 256 x D_I), whose fp32
 // accumulators alternate between the two 256-column halves of tensor memory, so the epilogue of one
 // overlaps the MMA of the next.  Warp roles: warp 0 issues TMA, warp 1 issues MMA (one thread each) and owns
-// the TMEM allocation, warps 2-9 are two epilogue groups (one per TMEM half).
+// the TMEM allocation, the other warps are two epilogue groups (one per TMEM half).  In score-matrix mode a group is
+// eight warps (two per TMEM lane quadrant, each reducing half of the slot's columns): with four epilogue warps per
+// scheduler one warp's wait for its tensor-memory load or its weights is covered by the others.  Candidate mode and
+// the ragged decode mode keep four warps per group.
 // Every wait is bounded; on a timeout the CTA reports JANUS_DEV_WAIT_TIMEOUT and winds down normally.
 #include "janus_common.cuh"
 #include "sm100_ptx.cuh"
@@ -22,7 +25,8 @@ using namespace ptx;
 
 constexpr int TC_KEYS = 128;        // keys per tile = MMA M
 constexpr int TC_N = 256;           // (token, head) rows per MMA = MMA N
-constexpr int TC_THREADS = 320;     // 1 TMA warp + 1 MMA warp + 8 epilogue warps
+constexpr int TC_THREADS = 320;     // candidate mode: 1 TMA warp + 1 MMA warp + 8 epilogue warps
+constexpr int TC_THREADS16 = 576;   // score-matrix mode: 16 epilogue warps, two per TMEM lane quadrant and slot, each takes half the columns
 constexpr int TC_THREADS_RAGGED = 192;   // ragged mode: one epilogue group (4 warps), so that four CTAs fit an SM
 constexpr int TC_SMEM_BUDGET = 227 * 1024;
 constexpr int TC_MAX_STAGES = 6;
@@ -113,7 +117,7 @@ __device__ __forceinline__ void reduce_chunk(const uint32_t (&r)[32], const floa
 }
 
 template <int H, bool FP8, bool CAND, bool RAGGED>
-__global__ void __launch_bounds__(RAGGED ? TC_THREADS_RAGGED : TC_THREADS, RAGGED ? 4 : 1)
+__global__ void __launch_bounds__(RAGGED ? TC_THREADS_RAGGED : ((CAND) ? TC_THREADS : TC_THREADS16), RAGGED ? 4 : 1)
 indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const TcParams p, const TcCandParams cp) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int TPS = TC_N / H;                      // tokens per query sub-tile
@@ -167,7 +171,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->q_full), 1);
         for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->tmem_full[s]), 1); mbar_init(smem_u32(&bars->tmem_empty[s]), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->tmem_full[s]), 1); mbar_init(smem_u32(&bars->tmem_empty[s]), (!CAND && !RAGGED) ? 8 : 4); }
         bars->aborted = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
@@ -178,7 +182,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         tmem_relinquish();
     }
     // per-column weights (w * q_scale) and per-token bias factors of this CTA
-    constexpr int NTHREADS = RAGGED ? TC_THREADS_RAGGED : TC_THREADS;
+    constexpr int NTHREADS = RAGGED ? TC_THREADS_RAGGED : (CAND ? TC_THREADS : TC_THREADS16);
     for (int n = threadIdx.x; n < nq * TC_N; n += NTHREADS) {
         const int t = t0 + n / H, h = n % H;
         float v = 0.f;
@@ -268,10 +272,12 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             if (!ok) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: warps 2..9
+        // ------------------------------------------------------------------ epilogue: warps 2 and up
         constexpr int NCHUNK = RAGGED ? H / 32 : TC_N / 32;   // 32-column chunks to reduce (ragged: the first query row only)
         static_assert(NCHUNK % 2 == 0, "chunks are processed in pairs");
-        const int e = (warp - 2) >> 2;          // epilogue group = TMEM half it drains
+        constexpr bool W16 = !CAND && !RAGGED;
+        const int e = ((warp - 2) >> 2) & 1;    // epilogue group = TMEM half it drains
+        const int chalf = W16 ? (warp - 2) >> 3 : 0;   // 16 warps: which half of the slot's columns
         const int quad = warp & 3;              // TMEM lanes 32*quad .. 32*quad+31
         const float neg_inf = __int_as_float(0xff800000);
         bool ok = true;
@@ -337,7 +343,28 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 };
                 // two register buffers: the load of the next 32 columns is in flight while this one is reduced
                 uint32_t ra[32], rb[32];
-                tmem_ld32_issue(taddr, ra);
+                constexpr int CPW = W16 ? NCHUNK / 2 : NCHUNK;       // chunks per warp
+                const int cbase = chalf * CPW;
+                tmem_ld32_issue(taddr + cbase * 32, ra);
+                if constexpr (W16) {
+#pragma unroll
+                for (int cc = 0; cc < CPW; cc += 2) {
+                    const int c = cbase + cc;
+                    tmem_ld_wait(ra);
+                    tmem_ld32_issue(taddr + (c + 1) * 32, rb);
+                    auto st = [&](int tt, float v) { store(tt + (cbase * 32) / H, v); };
+                    reduce_chunk<H>(ra, ws + j * TC_N + c * 32, cc * 32, acc, st);
+                    tmem_ld_wait(rb);
+                    if (cc + 2 < CPW) {
+                        tmem_ld32_issue(taddr + (c + 2) * 32, ra);
+                    } else {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[slot]));
+                    }
+                    reduce_chunk<H>(rb, ws + j * TC_N + (c + 1) * 32, (cc + 1) * 32, acc, st);
+                }
+                } else
 #pragma unroll
                 for (int c = 0; c < NCHUNK; c += 2) {
                     tmem_ld_wait(ra);
@@ -364,7 +391,7 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             }
         }
         // key tiles no token of this CTA may see: -inf (score-matrix mode only)
-        for (int tile = vis_end + e; !CAND && !RAGGED && tile < tile_end; tile += 2) {
+        for (int tile = vis_end + e; !CAND && !RAGGED && chalf == 0 && tile < tile_end; tile += 2) {
             const int64_t s = static_cast<int64_t>(tile) * TC_KEYS + quad * 32 + lane;
             if (s < p.n_keys)
                 for (int t = t0; t <= t_hi; ++t) p.scores[static_cast<int64_t>(t) * p.ld + s] = neg_inf;
@@ -427,7 +454,7 @@ template <int H, bool FP8, bool CAND, bool RAGGED = false>
 static int launch_tc(const CUtensorMap& tq, const CUtensorMap& tk, const TcParams& p, const TcCandParams& cp, dim3 grid, size_t smem,
                      cudaStream_t stream) {
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(indexer_tc_kernel<H, FP8, CAND, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    indexer_tc_kernel<H, FP8, CAND, RAGGED><<<grid, RAGGED ? TC_THREADS_RAGGED : TC_THREADS, smem, stream>>>(tq, tk, p, cp);
+    indexer_tc_kernel<H, FP8, CAND, RAGGED><<<grid, RAGGED ? TC_THREADS_RAGGED : (CAND ? TC_THREADS : TC_THREADS16), smem, stream>>>(tq, tk, p, cp);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }
