@@ -219,7 +219,11 @@ int janus_page_union(uint32_t* dst, const uint32_t* src, int64_t n_phys_pages, v
  * with an fp32 online softmax.  Token s lives at element offset
  *     page_table[s / page_size] * page_stride + (s % page_size) * tok_stride + h_kv * head_stride
  * of k_pool (keys, d_qk values) and v_pool (values, d_v values); query head h reads kv head h * n_kv_heads / H_q.
- * v_pool may alias k_pool (latent layout: the value is the first d_v dims of the key row).
+ * v_pool may alias k_pool (latent layout: the value is the first d_v dims of the key row; then d_v <= d_qk, else
+ * JANUS_ERR_INVALID_ARG).
+ * A selected token beyond the page table, or whose page table entry is negative, is skipped with
+ * JANUS_DEV_INDEX_OUT_OF_RANGE.  The upper end of the pool is not known to this call: a physical page id past the pool
+ * is NOT caught here.  janus_page_demand on the same idx and page table checks every id against n_phys_pages.
  *
  *   q     [M, H_q, d_qk] bf16, dense
  *   idx   [M, k] int32, -1 padded (any position); duplicates are attended twice
@@ -275,18 +279,21 @@ int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_siz
  *                              (no causal mask: the new token sees all of its session's keys).  q_idx [B, H_I, D_I]
  *                              contiguous, w [B, H_I], q_scale [B, H_I] or [H_I]; max_keys = an upper bound of the
  *                              longest session (host value, sizes the launch; at most total_keys, else
- *                              JANUS_ERR_INVALID_ARG); total_keys = rows of k_idx.
+ *                              JANUS_ERR_INVALID_ARG); total_keys = rows of k_idx.  A session whose offsets leave
+ *                              [0, total_keys] is cut back to the part inside with JANUS_DEV_INDEX_OUT_OF_RANGE.
  *                              Tensor-core path only: H_I = 64 and 128- or 256-byte rows, else JANUS_ERR_UNSUPPORTED.
  *                              dtype JANUS_DTYPE_FP8_Q_FP4_K: keys packed two per byte (D_I = 128, k_idx 32-byte aligned,
  *                              k_stride_tok a multiple of 64 elements), scales as for FP8.
  * janus_topk_batch             idx[b, 0:k) = top-k of the row_lengths[b] scores starting at scores[row_offsets[b]] (positions inside
  *                              the session, -1 padded), count / kth as in janus_topk.  row_offsets [B + 1] and row_lengths
  *                              [B] are int64 device arrays; row_lengths may be NULL (rows then run up to the next offset);
- *                              offsets are multiples of 4.
+ *                              offsets are multiples of 4.  A row whose offset is negative or not a multiple of 4, or whose
+ *                              length is negative, is left empty (idx -1, count 0) with JANUS_DEV_INDEX_OUT_OF_RANGE.
  * janus_page_demand_batch      janus_page_demand over all rows at once: row r marks page_tables[table_offsets[r] + s / page_size]
  *                              for its selected tokens s < demand_limits[r] (the session's cached history length) into one
  *                              bitmap over the global pool; lists, runs and the miss set against `predicted_bitmap` (for
- *                              decode: the pages already resident) as in janus_page_demand.
+ *                              decode: the pages already resident) as in janus_page_demand.  A negative table offset
+ *                              makes that row's table empty (its tokens are reported and skipped).
  * janus_sparse_attn_decode     janus_sparse_attn_prefill with one query row per session and per-row page tables.
  */
 int janus_indexer_scores_batch(const void* q_idx, const void* k_idx, int64_t k_stride_tok,
@@ -317,6 +324,26 @@ int janus_sparse_attn_decode(const void* q, int B, int H_q, int d_qk,
                              const int32_t* page_tables, const int64_t* table_offsets,
                              float softmax_scale, void* out, float* lse,
                              int32_t* dev_status, void* stream);
+
+/*
+ * Diagnostics.  The paper has no counterpart for either call.
+ *
+ * janus_selftest_bounded_wait   Every wait inside the tensor-core kernels (on an mbarrier: a copy that has not landed, a
+ *                               tensor-memory slot that is not free) gives up after a fixed number of polls, writes
+ *                               JANUS_DEV_WAIT_TIMEOUT to *dev_status and lets the kernel return normally.  This call runs
+ *                               that wait on a barrier nobody arrives on, with `max_polls` polls (1 .. 65536), so that the
+ *                               time-out path can be exercised without a broken pipeline: afterwards *dev_status is
+ *                               JANUS_DEV_WAIT_TIMEOUT, *elapsed_ns (device int64, may be NULL) holds how long the wait
+ *                               took, and the context is as usable as before.
+ * janus_fp8_mma_probe           Launches `n_ctas` CTAs (one per SM is the intended use) that each issue `fills_per_cta`
+ *                               dense FP8 E4M3 tensor-core accumulator fills (M = 128, N = 256, K = 128; operands in shared
+ *                               memory, nothing else in the kernel) and writes the launch's flop count to *flop_per_launch
+ *                               (host double, may be NULL).  Timed by the caller with events on `stream`, it gives the FP8
+ *                               tensor rate this GPU sustains under its power limit: the denominator of the indexer's
+ *                               roofline fraction.  Asynchronous; uses no device memory besides *dev_status.
+ */
+int janus_selftest_bounded_wait(int max_polls, int64_t* elapsed_ns, int32_t* dev_status, void* stream);
+int janus_fp8_mma_probe(int n_ctas, int fills_per_cta, double* flop_per_launch /* host */, int32_t* dev_status, void* stream);
 
 #ifdef __cplusplus
 }

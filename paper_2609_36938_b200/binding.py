@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from typing import Dict, Optional
+from typing import Dict, Optional, Tuple
 
 import torch
 
@@ -19,6 +19,7 @@ JANUS_OK = 0
 ERR_NAMES = {1: "JANUS_ERR_INVALID_ARG", 2: "JANUS_ERR_UNSUPPORTED", 3: "JANUS_ERR_WORKSPACE_TOO_SMALL", 4: "JANUS_ERR_CUDA"}
 DEV_NAMES = {101: "JANUS_DEV_INDEX_OUT_OF_RANGE", 102: "JANUS_DEV_CAPACITY_EXCEEDED", 103: "JANUS_DEV_WAIT_TIMEOUT"}
 DTYPE_BF16, DTYPE_FP8_E4M3, DTYPE_FP8_Q_FP4_K = 0, 1, 2
+MBAR_MAX_POLLS = 1 << 16      # the kernels' limit on polls of one in-kernel wait (csrc/sm100_ptx.cuh)
 
 # every symbol include/janus.h declares
 EXPORTS = [
@@ -30,6 +31,7 @@ EXPORTS = [
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
     "janus_indexer_scores_batch", "janus_topk_batch", "janus_page_demand_batch", "janus_sparse_attn_decode",
     "janus_topk_entries", "janus_entry_expand",
+    "janus_selftest_bounded_wait", "janus_fp8_mma_probe",
 ]
 
 
@@ -94,6 +96,10 @@ def load() -> ctypes.CDLL:
     lib.janus_topk_entries.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_p]
     lib.janus_entry_expand.restype = c_i
     lib.janus_entry_expand.argtypes = [c_p, c_i, c_i, c_i, c_i64, c_p, c_p]
+    lib.janus_selftest_bounded_wait.restype = c_i
+    lib.janus_selftest_bounded_wait.argtypes = [c_i, c_p, c_p, c_p]
+    lib.janus_fp8_mma_probe.restype = c_i
+    lib.janus_fp8_mma_probe.argtypes = [c_i, c_i, ctypes.POINTER(ctypes.c_double), c_p, c_p]
     _lib = lib
     return lib
 
@@ -417,6 +423,26 @@ def janus_sparse_attn_decode(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torc
                                       float(softmax_scale), _ptr(out), _ptr(lse), _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_sparse_attn_decode")
     return out, lse
+
+
+# ---- diagnostics ---------------------------------------------------------------------------------------------------
+def janus_selftest_bounded_wait(max_polls: int = 256) -> Tuple[int, float]:
+    """Runs the kernels' bounded wait on a barrier nobody arrives on.  Returns (status word afterwards, seconds the wait took);
+    the status word is cleared again."""
+    st = dev_status_tensor()
+    st.zero_()
+    ns = torch.zeros(1, dtype=torch.int64, device=st.device)
+    _check(load().janus_selftest_bounded_wait(int(max_polls), _ptr(ns), _ptr(st), _stream()), "janus_selftest_bounded_wait")
+    v = int(st.item())
+    st.zero_()
+    return v, float(ns.item()) * 1e-9
+
+
+def janus_fp8_mma_probe(n_ctas: int, fills_per_cta: int) -> float:
+    """Launches the dense FP8 tensor-rate probe on the current stream; returns the launch's flop count."""
+    flop = ctypes.c_double(0.0)
+    _check(load().janus_fp8_mma_probe(int(n_ctas), int(fills_per_cta), ctypes.byref(flop), _ptr(dev_status_tensor()), _stream()), "janus_fp8_mma_probe")
+    return flop.value
 
 
 # ---- helpers to move generator output (bit patterns) onto the device -------------------------------------------

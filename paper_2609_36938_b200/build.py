@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libjanus.so")
 SOURCES = ["janus_api.cu", "indexer_generic.cu", "indexer_tc.cu", "topk.cu", "page_demand.cu", "sparse_attn_generic.cu",
-           "sparse_attn_latent_pair.cu", "indexer_topk.cu"]
+           "sparse_attn_latent_pair.cu", "indexer_topk.cu", "diagnostics.cu"]
 
 
 def _nvcc() -> str:

@@ -78,6 +78,7 @@ struct TcBarriers {
     uint64_t k_empty[TC_MAX_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t mma_drain;       // abort path only: every MMA issued so far has completed
     uint32_t tmem_base;
     int aborted;
 };
@@ -146,7 +147,14 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         t0 = blockIdx.y;                                        // one query row per grid row; the sub-tile's other rows are not stored
         key_base = cp.key_offsets[blockIdx.y];
         key_count = cp.key_offsets[blockIdx.y + 1] - key_base;
-        if (key_count < 0) key_count = 0;
+        // the offsets come from device memory: a session that lies outside the key array (p.n_keys rows) is reported and cut
+        // back to the part inside it, so that neither the per-key scale / bias reads nor the score writes leave their arrays
+        if (key_base < 0 || key_count < 0 || key_base > p.n_keys || key_count > p.n_keys - key_base) {
+            if (threadIdx.x == 0) report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
+            if (key_base < 0 || key_base > p.n_keys) { key_base = 0; key_count = 0; }
+            if (key_count < 0) key_count = 0;
+            if (key_count > p.n_keys - key_base) key_count = p.n_keys - key_base;
+        }
         n_tiles = static_cast<int>((key_count + TC_KEYS - 1) / TC_KEYS);
     }
     const int t_hi = min(p.M, t0 + tpc) - 1;                    // last real token of this CTA
@@ -165,14 +173,14 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         if (threadIdx.x == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
         return;
     }
-    // an earlier CTA of this launch gave up on a wait: do not start new work on a broken pipeline
-    if (p.dev_status != nullptr && *reinterpret_cast<volatile int32_t*>(p.dev_status) == JANUS_DEV_WAIT_TIMEOUT) return;
-
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->q_full), 1);
         for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bars->tmem_full[s]), 1); mbar_init(smem_u32(&bars->tmem_empty[s]), (!CAND && !RAGGED) ? 8 : 4); }
-        bars->aborted = 0;
+        mbar_init(smem_u32(&bars->mma_drain), 1);
+        // an earlier CTA of this launch gave up on a wait: this one starts no work on a broken pipeline.  One thread reads the
+        // status word and the whole CTA follows that one reading (a second reading could differ and split the roles).
+        bars->aborted = (p.dev_status != nullptr && *reinterpret_cast<volatile int32_t*>(p.dev_status) == JANUS_DEV_WAIT_TIMEOUT) ? 1 : 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
@@ -201,8 +209,11 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     volatile int* aborted = &bars->aborted;
+    const bool run = *aborted == 0;       // read once, after the barrier: the same value in every thread
 
-    if (warp == 0) {
+    if (!run) {
+        // nothing to do: tensor memory goes back below
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && n_vis > 0) {
             const int atom_elems = FP8 ? 128 : 64;
@@ -269,7 +280,13 @@ indexer_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 if (!ok) break;
                 umma_commit(smem_u32(&bars->k_empty[s]));
             }
-            if (!ok) { *aborted = 1; report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT); }
+            if (!ok) {
+                *aborted = 1;
+                report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
+                // tensor memory is freed after the barrier below: the instructions already issued finish first
+                umma_commit(smem_u32(&bars->mma_drain));
+                mbar_wait(smem_u32(&bars->mma_drain), 0);
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue: warps 2 and up

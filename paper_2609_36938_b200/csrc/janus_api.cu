@@ -1,7 +1,5 @@
 // Entry points that validate arguments and pick a kernel: janus_indexer_scores, janus_sparse_attn_prefill,
 // plus the version / error queries.  janus_topk and janus_page_demand live beside their kernels.
-#include <cstdlib>
-
 #include "janus_common.cuh"
 
 namespace janus {
@@ -86,9 +84,7 @@ extern "C" int janus_indexer_scores(const void* q_idx, int64_t q_stride_tok, con
     if (M == 0 || n_keys == 0) return JANUS_OK;
     if (!scores || !aligned16(scores)) return JANUS_ERR_INVALID_ARG;
     if (scores_ld < n_keys || (scores_ld & 3) != 0) return JANUS_ERR_INVALID_ARG;
-    // debugging aid: JANUS_FORCE_GENERAL_INDEXER=1 routes every shape to the general kernel
-    const char* force_general = getenv("JANUS_FORCE_GENERAL_INDEXER");
-    if (!(force_general && force_general[0] == '1') && indexer_tc_supported(M, H_I, D_I, n_keys, q_stride_tok, k_stride_tok, dtype))
+    if (indexer_tc_supported(M, H_I, D_I, n_keys, q_stride_tok, k_stride_tok, dtype))
         return launch_indexer_tc(q_idx, k_idx, k_stride_tok, w, q_scale, q_scale_stride_tok, k_scale, row_bias, col_bias, M, H_I, D_I,
                                  n_keys, q_pos0, causal, dtype, scores, scores_ld, dev_status, stream);
     if (dtype == JANUS_DTYPE_FP8_Q_FP4_K) return JANUS_ERR_UNSUPPORTED;   // 4-bit keys: tensor-core shapes only
@@ -132,10 +128,9 @@ static int sparse_attn_dispatch(const void* q, int M, int H_q, int d_qk, const v
     if (!q || !k_pool || !v_pool || !out || !page_table || (k > 0 && !idx)) return JANUS_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(out)) return JANUS_ERR_INVALID_ARG;
     if ((page_stride % 8) != 0 || (tok_stride % 8) != 0 || (head_stride % 8) != 0) return JANUS_ERR_INVALID_ARG;
+    if (v_pool == k_pool && d_v > d_qk) return JANUS_ERR_INVALID_ARG;   // an aliased value row is a prefix of the key row
     if (M > 2147483647 / 2) return JANUS_ERR_UNSUPPORTED;
-    // debugging aid: JANUS_FORCE_GENERAL_ATTN=1 routes every shape to the general kernel
-    const char* force_general = getenv("JANUS_FORCE_GENERAL_ATTN");
-    if (!(force_general && force_general[0] == '1') && softmax_scale > 0.f &&
+    if (softmax_scale > 0.f &&
         sparse_attn_latent_tc_supported(M, H_q, d_qk, k_pool, v_pool, page_stride, tok_stride, n_kv_heads, d_v, k))
         return launch_sparse_attn_latent_tc(q, M, k_pool, page_stride, tok_stride, idx, k, page_size, page_table, n_logical_pages,
                                             table_offsets, softmax_scale, out, lse, dev_status, stream);

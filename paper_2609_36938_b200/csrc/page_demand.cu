@@ -238,8 +238,9 @@ page_mark_rows_kernel(const int32_t* __restrict__ idx, int64_t n_rows, int k, co
     for (int64_t e = static_cast<int64_t>(blockIdx.x) * MARK_THREADS + threadIdx.x; e < n_idx; e += stride) {
         const int64_t r = e / k;
         const int64_t off = __ldg(table_offsets + r);
-        mark_one(__ldg(idx + e), __ldg(demand_limits + r), page_size, page_shift, page_tables + off, __ldg(table_offsets + r + 1) - off,
-                 n_phys_pages, bitmap, dev_status);
+        // a table that starts before the array has no pages: its selected tokens are reported and skipped
+        mark_one(__ldg(idx + e), __ldg(demand_limits + r), page_size, page_shift, page_tables + (off < 0 ? 0 : off),
+                 off < 0 ? 0 : __ldg(table_offsets + r + 1) - off, n_phys_pages, bitmap, dev_status);
     }
 }
 

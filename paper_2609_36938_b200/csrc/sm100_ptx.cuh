@@ -45,9 +45,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) { 
         : "memory");
     return ok != 0;
 }
-// Bounded wait: one cheap probe first (the common case in a running pipeline), then up to `max_polls` blocking polls
-// (each poll itself blocks for a short, hardware-chosen time).  Returns false if the phase never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = (1u << 22)) {
+// Limit of one wait, in polls.  A blocking poll that fails returns after a hardware-chosen time (measured here by the
+// library's self-test export: about four microseconds), so a wait on a phase that never completes gives up after a
+// quarter of a second; the longest wait of a healthy pipeline (a CTA's first operand tile, a few microseconds; a peer CTA
+// that is one 64-key tile behind) is thousands of times shorter.
+constexpr uint32_t MBAR_MAX_POLLS = 1u << 16;
+// Bounded wait: one cheap probe first (the common case in a running pipeline), then up to `max_polls` blocking polls.
+// Returns false if the phase never completed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = MBAR_MAX_POLLS) {
     if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < max_polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
@@ -334,7 +339,7 @@ __device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_add
     asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // Bounded wait on a local mbarrier that peers arrive on (acquire at cluster scope).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t max_polls = (1u << 22)) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t max_polls = MBAR_MAX_POLLS) {
     for (uint32_t i = 0; i < max_polls; ++i) {
         uint32_t ok;
         asm volatile(

@@ -32,8 +32,10 @@ sparse_attn_generic_kernel(const uint16_t* __restrict__ q, int M, int H_q, int d
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int t = blockIdx.x;
     if (table_offsets != nullptr) {     // every row has a page table of its own (a batch of sessions)
-        page_table += table_offsets[t];
-        n_logical_pages = table_offsets[t + 1] - table_offsets[t];
+        const int64_t tbl = table_offsets[t];
+        n_logical_pages = table_offsets[t + 1] - tbl;
+        if (tbl < 0) n_logical_pages = 0;          // a table that starts before the array: every selected token is reported and skipped
+        else page_table += tbl;
     }
     const int heads_per_kv = H_q / n_kv_heads;
     const int groups_per_kv = (heads_per_kv + G - 1) / G;
@@ -61,7 +63,8 @@ sparse_attn_generic_kernel(const uint16_t* __restrict__ q, int M, int H_q, int d
         __syncthreads();
         if (tid < AG_KT) {
             int s = base + tid < k ? my_idx[base + tid] : -1;
-            if (s >= 0 && s / page_size >= n_logical_pages) { report(dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE); s = -1; }
+            // a token beyond the page table, or a negative physical page id in it, is reported and skipped
+            if (s >= 0 && (s / page_size >= n_logical_pages || __ldg(page_table + s / page_size) < 0)) { report(dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE); s = -1; }
             srow[tid] = s;
         }
         __syncthreads();

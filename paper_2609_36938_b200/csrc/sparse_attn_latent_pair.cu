@@ -78,9 +78,6 @@ struct LpShared {
     uint64_t x_full[2];                           // the peer's partial logits of the tile using logit buffer b have arrived
     uint64_t x_empty[2];                          // the PEER has read this CTA's previous partial logits out of its exchange buffer b
     uint32_t vmask[LP_SLOTS];
-#ifdef JANUS_ATTN_PROFILE
-    long long prof_ts[2], prof_ts2[2];            // when the exchange warps saw the logits complete / had sent them
-#endif
     uint32_t tmem_base;
     uint32_t start_abort[2];
 };
@@ -101,25 +98,6 @@ struct LpParams {
     int M;
     int32_t* dev_status;
 };
-
-// Optional per-role cycle accounting for tuning (off in the product build): with -DJANUS_ATTN_PROFILE the lse output of
-// token t receives, instead of the log-sum-exp, the cycles each role of CTA 0 spent in total and inside its waits.
-#ifdef JANUS_ATTN_PROFILE
-#define LP_PROF_DECL(name) long long name = 0
-#define LP_PROF_WAIT(acc, expr) ([&] { const long long _t0 = clock64(); const bool _r = (expr); acc += clock64() - _t0; return _r; }())
-#define LP_PROF_NOW() clock64()
-#define LP_PROF_SEG(acc, t_prev) do { const long long _n = clock64(); acc += _n - t_prev; t_prev = _n; } while (0)
-#ifndef JANUS_PROF_CTA
-#define JANUS_PROF_CTA 0u
-#endif
-#define LP_PROF_PUT(slot, v) do { if (p.lse != nullptr && c == JANUS_PROF_CTA) p.lse[static_cast<int64_t>(cid) * LP_HEADS + (slot)] = static_cast<float>(v); } while (0)
-#else
-#define LP_PROF_DECL(name)
-#define LP_PROF_WAIT(acc, expr) (expr)
-#define LP_PROF_NOW() 0
-#define LP_PROF_SEG(acc, t_prev) do { } while (0)
-#define LP_PROF_PUT(slot, v) do { } while (0)
-#endif
 
 __device__ __forceinline__ float lp_exp2(float x) {   // ex2.approx: 2 ulp, exp2(-inf) = 0
     float y;
@@ -206,15 +184,14 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (n_my > 0) fetch_q(0);
             constexpr uint32_t idesc_qk = umma_idesc_major(1u, LP_HEADS, LP_TILE, 0u, 0u);
             constexpr uint32_t idesc_pv = umma_idesc_major(1u, LP_HEADS, LP_DVH, 0u, 1u);
-            LP_PROF_DECL(w_kfull); LP_PROF_DECL(w_pfull); LP_PROF_DECL(w_q);
-            const long long prof_t0 = LP_PROF_NOW();
+
             const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem), 16);
             const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem), 16);
             const uint32_t v_lo = umma_desc_lo(smem_u32(k_smem), LP_K_ATOM_BYTES);     // value half = first four owned atoms
             bool ok = true;
             int s_next = 0, pv_next = 0;                 // next logit tile / next P.V to issue, counted over all tokens
             for (int it = 0; it < n_my && ok; ++it) {
-                ok = LP_PROF_WAIT(w_q, mbar_wait(qf, static_cast<uint32_t>(it) & 1u) && mbar_wait(smem_u32(&sh->qt_full), static_cast<uint32_t>(it) & 1u));
+                ok = (mbar_wait(qf, static_cast<uint32_t>(it) & 1u) && mbar_wait(smem_u32(&sh->qt_full), static_cast<uint32_t>(it) & 1u));
                 if (!ok) break;
                 tc_fence_after();
                 const int tok_begin = it * n_tiles, tok_end = tok_begin + n_tiles;
@@ -258,7 +235,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                         umma_commit(smem_u32(&sh->s_full[b]));
                         ++s_next;
                         idle = 0;
-                    } else if (++idle > (1u << 24)) {     // nothing became ready for about a second: give up
+                    } else if (++idle > (1u << 21)) {     // nothing became ready for some two million probes (a few tenths of a second): give up
                         ok = false;
                         break;
                     }
@@ -269,7 +246,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                 if (it + 1 < n_my) fetch_q(it + 1);
             }
             if (!ok) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
-            LP_PROF_PUT(0, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(1, w_kfull); LP_PROF_PUT(2, w_pfull); LP_PROF_PUT(9, w_q);
         }
         __syncwarp();
     } else if (warp <= LP_GATHER_WARPS) {
@@ -283,8 +259,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const uint32_t g_sw0 = static_cast<uint32_t>((g_sub ^ g_rr) << 4), g_sw1 = static_cast<uint32_t>((g_sub ^ (4 + g_rr)) << 4);   // even / odd q
         const int64_t seg_off = 512 * static_cast<int64_t>(c); // first owned byte of a row
         bool ok = true;
-        LP_PROF_DECL(w_kempty); LP_PROF_DECL(w_group);
-        const long long prof_t0 = LP_PROF_NOW();
+
         int64_t tbl_nxt = 0, tbl_n_nxt = p.n_logical_pages;     // page table (start, length) of the query row the last load_raw was for
         auto load_raw = [&](int gh) -> int {                   // lane r owns row r of global half-tile gh
             if (gh >= total_half) return -1;
@@ -294,6 +269,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (p.table_offsets != nullptr) {                  // every query row has a page table of its own (a batch of sessions)
                 tbl_nxt = __ldg(p.table_offsets + t_row);
                 tbl_n_nxt = __ldg(p.table_offsets + t_row + 1) - tbl_nxt;
+                if (tbl_nxt < 0) tbl_n_nxt = 0;                // a table that starts before the array: its tokens are reported and skipped
             }
             return slot < p.k ? __ldg(p.idx + t_row * p.k + slot) : -1;
         };
@@ -303,10 +279,11 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (s_tok >= 0) {
                 const int64_t lp = p.page_shift >= 0 ? (s_tok >> p.page_shift) : (s_tok / p.page_size);
                 const int within = p.page_shift >= 0 ? (s_tok & (p.page_size - 1)) : (s_tok % p.page_size);
-                if (lp >= tbl_n) {
+                const int32_t phys = lp < tbl_n ? __ldg(p.page_table + tbl + lp) : -1;
+                if (phys < 0) {     // beyond the page table, or a negative physical page id in it
                     report(p.dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
                 } else {
-                    ptr += (static_cast<int64_t>(__ldg(p.page_table + tbl + lp)) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
+                    ptr += (static_cast<int64_t>(phys) * p.page_stride + static_cast<int64_t>(within) * p.tok_stride) * 2;
                     valid = true;
                 }
             }
@@ -328,7 +305,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             const bool s_ok = valid_cur;
             const uint32_t valid_mask = __ballot_sync(0xffffffffu, s_ok);
             // the tile buffer must have been released by the P.V three tiles back
-            ok = LP_PROF_WAIT(w_kempty, mbar_wait(smem_u32(&sh->k_empty[buf]), (static_cast<uint32_t>((hi >> 1) / LP_BUFS) & 1u) ^ 1u));
+            ok = (mbar_wait(smem_u32(&sh->k_empty[buf]), (static_cast<uint32_t>((hi >> 1) / LP_BUFS) & 1u) ^ 1u));
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (lane == 0) sh->vmask[2 * buf + hf] = valid_mask;
@@ -353,7 +330,7 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             cp_async_commit();
             row_nxt = resolve(raw_nxt, tbl_nxt, tbl_n_nxt, valid_nxt);   // page-table load overlaps the copies in flight
             raw_nxt = load_raw(next_owned(hi_nxt));
-            LP_PROF_WAIT(w_group, (cp_async_wait<0>(), true));
+            cp_async_wait<0>();
             fence_proxy_async();              // publish the landed rows to the MMA (async) proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->k_full[buf]));
@@ -361,7 +338,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             valid_cur = valid_nxt;
         }
         if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
-        if (g == 0 && lane == 0) { LP_PROF_PUT(3, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(4, w_kempty); LP_PROF_PUT(5, w_group); }
     } else if (warp < LP_SMAX_WARP0) {
         // ================================================================== exchange: partial logits -> the peer's buffer
         const int quad = warp & 3;                         // warps 4..7 -> TMEM lane quadrants 0..3
@@ -404,9 +380,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-#ifdef JANUS_ATTN_PROFILE
-            if (warp == LP_XCHG_WARP0 && lane == 0) sh->prof_ts[b] = clock64();
-#endif
             const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
             uint32_t r0[32], r1[32];
             tmem_ld32_issue(s_addr, r0);
@@ -440,9 +413,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                                        __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 2]), __uint_as_float(r1[8 * j8 + 3]))),
                                        __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 4]), __uint_as_float(r1[8 * j8 + 5]))),
                                        __uint_as_float(lp_pack_f16x2(__uint_as_float(r1[8 * j8 + 6]), __uint_as_float(r1[8 * j8 + 7]))), bar);
-#ifdef JANUS_ATTN_PROFILE
-            if (warp == LP_XCHG_WARP0 && lane == 0) sh->prof_ts2[b] = clock64();
-#endif
         }
             // the token's last logit tile is complete, so nothing reads its queries any more: bring in the next token's
             if (ok && it + 1 < n_my) load_q(it + 1);
@@ -456,12 +426,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
         const float neg_inf = __int_as_float(0xff800000);
         const bool out_al32 = (reinterpret_cast<uint64_t>(p.out) & 31u) == 0u;
         bool ok = true;
-        LP_PROF_DECL(w_sfull); LP_PROF_DECL(w_xfull); LP_PROF_DECL(w_send);
-        LP_PROF_DECL(e_wait); LP_PROF_DECL(e_out); LP_PROF_DECL(w_x01); LP_PROF_DECL(w_s01); LP_PROF_DECL(x_lat); LP_PROF_DECL(x_lat2);
-        LP_PROF_DECL(s_ld); LP_PROF_DECL(s_peer); LP_PROF_DECL(s_arr); LP_PROF_DECL(s_exp); LP_PROF_DECL(s_st);
-        const long long prof_t0 = LP_PROF_NOW();
-        long long seg = prof_t0;
-        (void)seg;
         const uint32_t peer_xempty = mapa_shared(smem_u32(&sh->x_empty[0]), peer);
         int gi = 0;                 // tiles done so far, over all tokens
         for (int it = 0; it < n_my && ok; ++it) {
@@ -475,17 +439,12 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             if (warp == LP_SMAX_WARP0 && lane == 0) mbar_expect_tx(smem_u32(&sh->x_full[b]), LP_XBUF_BYTES);
             // k_full is complete long before s_full; waiting on it as well makes the validity masks written by the gather
             // warps visible to this thread directly rather than through the MMA warp
-#ifdef JANUS_ATTN_PROFILE
-            { const long long _t0 = clock64(); ok = mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s); const long long _d = clock64() - _t0; w_sfull += _d; if (i < 2) w_s01 += _d; }
-#else
             ok = mbar_wait(smem_u32(&sh->k_full[buf]), ph_k) && mbar_wait(smem_u32(&sh->s_full[b]), ph_s);
-#endif
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t s_addr = lane_addr + LP_COL_S + b * LP_TILE;
             float2 x[LP_TILE / 2];          // logits of keys 2j, 2j+1
-            seg = LP_PROF_NOW();
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t r[32];
@@ -497,18 +456,11 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
-            LP_PROF_SEG(s_ld, seg);
             // the peer's partial logits of the same tile (bytes counted as they land: visible once the phase completes)
-#ifdef JANUS_ATTN_PROFILE
-            { const long long _t0 = clock64(); ok = mbar_wait(smem_u32(&sh->x_full[b]), ph_s); const long long _n = clock64(); const long long _d = _n - _t0; w_xfull += _d; if (i < 2) w_x01 += _d;
-              if (_d > 100) { x_lat += _n - *reinterpret_cast<volatile long long*>(&sh->prof_ts[b]); x_lat2 += _n - *reinterpret_cast<volatile long long*>(&sh->prof_ts2[b]); } }
-#else
             ok = mbar_wait(smem_u32(&sh->x_full[b]), ph_s);
-#endif
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             float tile_max = neg_inf;
-            seg = LP_PROF_NOW();
             {
                 const uint4* xin = reinterpret_cast<const uint4*>(xbuf + b * LP_XBUF_BYTES) + h;
 #pragma unroll
@@ -537,11 +489,9 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                 }
                 tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             }
-            LP_PROF_SEG(s_peer, seg);
             // the exchange buffer has been read: the peer may send the tile after next into it
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster_relaxed(peer_xempty + static_cast<uint32_t>(b * 8));
-            LP_PROF_SEG(s_arr, seg);
             tile_max *= p.scale_log2e;                       // softmax_scale > 0
             // move the reference maximum only when this tile exceeds it by more than 2^8 (or on first use)
             float corr = 1.f;
@@ -583,7 +533,6 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             const float2 t4 = fadd2(t01, t23);
             const float tile_sum = t4.x + t4.y;
             l_sum += tile_sum;
-            LP_PROF_SEG(s_exp, seg);
             // P has one buffer: the previous tile's P.V must have completed
             if (gi > 0) {
                 ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
@@ -595,17 +544,14 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->p_full));
-            LP_PROF_SEG(s_st, seg);
         }
         if (!ok) break;
-        seg = LP_PROF_NOW();
         // ---- output: wait for the token's last P.V, normalise, round to bf16.  The next token's first P is produced by
         // these same warps afterwards, so its P.V cannot overwrite O before O has been read here.
         ok = mbar_wait(smem_u32(&sh->k_empty[(gi - 1) % LP_BUFS]), static_cast<uint32_t>((gi - 1) / LP_BUFS) & 1u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        LP_PROF_SEG(e_wait, seg);
         const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
         const bool have_o = __any_sync(0xffffffffu, l_sum > 0.f);   // some P.V of this token has written O
         uint16_t* orow = p.out + (static_cast<int64_t>(t) * LP_HEADS + h) * LP_DV + c * LP_DVH;
@@ -630,16 +576,10 @@ sparse_attn_latent_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const
                 for (int v = 0; v < 4; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
             }
         }
-        LP_PROF_SEG(e_out, seg);
-#ifndef JANUS_ATTN_PROFILE
         if (p.lse != nullptr && c == 0u)
             p.lse[static_cast<int64_t>(t) * LP_HEADS + h] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : neg_inf;
-#endif
         }
         if (!ok && lane == 0) report(p.dev_status, JANUS_DEV_WAIT_TIMEOUT);
-#ifdef JANUS_ATTN_PROFILE
-        if (warp == LP_SMAX_WARP0 && lane == 0) { LP_PROF_PUT(6, LP_PROF_NOW() - prof_t0); LP_PROF_PUT(7, w_sfull); LP_PROF_PUT(8, w_xfull); LP_PROF_PUT(10, w_send); LP_PROF_PUT(11, s_ld); LP_PROF_PUT(12, s_peer); LP_PROF_PUT(13, s_arr); LP_PROF_PUT(14, s_exp); LP_PROF_PUT(15, s_st); LP_PROF_PUT(16, e_wait); LP_PROF_PUT(17, e_out); LP_PROF_PUT(18, w_x01); LP_PROF_PUT(19, w_s01); LP_PROF_PUT(20, x_lat); LP_PROF_PUT(21, x_lat2); }
-#endif
     }
     tc_fence_before();
     __syncthreads();

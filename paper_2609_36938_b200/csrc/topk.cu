@@ -74,15 +74,24 @@ __global__ void entry_expand_kernel(const int32_t* __restrict__ idx_e, int M, in
 template <int CAP>
 __global__ void __launch_bounds__(TK_THREADS)
 topk_ragged_kernel(const float* __restrict__ scores, const int64_t* __restrict__ row_offsets, const int64_t* __restrict__ row_lengths, int k,
-                   int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth) {
+                   int32_t* __restrict__ idx, int32_t* __restrict__ count, float* __restrict__ kth, int32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using TopkShared = TopkSharedT<CAP>;
     TopkShared& sh = *reinterpret_cast<TopkShared*>(smem_raw);
     const int b = blockIdx.x;
     const int64_t off = row_offsets[b];
-    int64_t n = row_lengths != nullptr ? row_lengths[b] : row_offsets[b + 1] - off;
-    if (n < 0) n = 0;
-    if (n > 2147483639) n = 2147483639;
+    const int64_t n = row_lengths != nullptr ? row_lengths[b] : row_offsets[b + 1] - off;
+    // the offsets come from device memory: a row that starts before the array, off a 16-byte boundary (the row is read with
+    // 16-byte loads) or has a negative or unrepresentable length is reported and left empty, never read
+    if (off < 0 || (off & 3) != 0 || n < 0 || n > 2147483639) {
+        for (int i = threadIdx.x; i < k; i += blockDim.x) idx[static_cast<int64_t>(b) * k + i] = -1;
+        if (threadIdx.x == 0) {
+            if (count != nullptr) count[b] = 0;
+            if (kth != nullptr) kth[b] = __int_as_float(0xff800000);
+            report(dev_status, JANUS_DEV_INDEX_OUT_OF_RANGE);
+        }
+        return;
+    }
     topk_row(scores + off, static_cast<int>(n), k, b, idx + static_cast<int64_t>(b) * k, count, kth, sh);
 }
 
@@ -121,7 +130,7 @@ extern "C" int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, in
 }
 
 extern "C" int janus_topk_batch(const float* scores, const int64_t* row_offsets, const int64_t* row_lengths, int B, int k, int32_t* idx,
-                                int32_t* count, float* kth, int32_t* /*dev_status*/, void* stream_) {
+                                int32_t* count, float* kth, int32_t* dev_status, void* stream_) {
     using namespace janus;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (B < 0 || k <= 0) return JANUS_ERR_INVALID_ARG;
@@ -130,7 +139,7 @@ extern "C" int janus_topk_batch(const float* scores, const int64_t* row_offsets,
     // row lengths live on the device: the large candidate buffer serves any length
     const size_t smem = sizeof(TopkSharedT<TK_CAP>);
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_ragged_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    topk_ragged_kernel<TK_CAP><<<B, TK_THREADS, smem, stream>>>(scores, row_offsets, row_lengths, k, idx, count, kth);
+    topk_ragged_kernel<TK_CAP><<<B, TK_THREADS, smem, stream>>>(scores, row_offsets, row_lengths, k, idx, count, kth, dev_status);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }

@@ -85,6 +85,7 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     assert at(d_v=1024) == UNSUPPORTED
     assert at(tok_stride=1001) == INVALID
     assert at(q=None) == INVALID
+    assert at(d_qk=64, d_v=128) == INVALID                # k_pool == v_pool here: an aliased value row cannot be wider than the key row
 
 
 def test_binding_refuses_host_tensors_and_missing_library(monkeypatch):

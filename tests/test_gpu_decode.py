@@ -176,3 +176,108 @@ def test_prefill_indexer_and_selection_with_fp4_keys():
     rc = lib.janus_indexer_scores(qd.data_ptr(), 5 * D, kd.data_ptr(), D, wd.data_ptr(), args["q_scale"].data_ptr(), 5, args["k_scale"].data_ptr(),
                                   None, None, 3, 5, D, 64, 0, 1, 2, sc.data_ptr(), 64, None, 0, None, None)
     assert rc == 2                                            # JANUS_ERR_UNSUPPORTED
+
+
+def _status_word():
+    """Reads and clears the device status word (the tests below expect it to be set)."""
+    st = B.dev_status_tensor()
+    v = int(st.item())
+    st.zero_()
+    return v
+
+
+def test_batch_entries_report_and_skip_bad_offsets():
+    """Offsets and page ids that come from device memory are never trusted (the library's rule: device-visible conditions are
+    reported in the status word and skipped, nothing traps): a misaligned or negative score-row offset, a session that
+    leaves the key array, a negative page-table offset and a negative physical page id each set
+    JANUS_DEV_INDEX_OUT_OF_RANGE, leave the other rows' results as they are, and the next ordinary call passes."""
+    lengths = [900, 400, 2500, 131]
+    k, page, d_qk, d_v, H_q = 64, 64, 576, 512, 128
+    b = make_batch(23, lengths, "fp8", page=page)
+    nb = len(lengths)
+    dev = lambda x, kind: B.to_device(x, kind)
+    key_off = torch.from_numpy(b["key_off"]).cuda()
+    kd, qd, wd = dev(b["k"], "fp8"), dev(b["q"], "fp8"), dev(b["w"], "f32")
+    qs, ks = dev(b["q_scale"], "f32"), dev(b["k_scale"], "f32")
+    total = b["k"].shape[0]
+    good = B.janus_indexer_scores_batch(qd, kd, wd, key_off, max(lengths) + 4, q_scale=qs, k_scale=ks)
+    B.check_dev_status()
+    row_len = torch.tensor([L + 1 for L in lengths], dtype=torch.int64, device="cuda")
+    idx_good, cnt_good, _ = B.janus_topk_batch(good, key_off, k, row_lengths=row_len)
+    B.check_dev_status()
+
+    # ---- janus_topk_batch: row 1 starts off a 16-byte boundary, row 3 before the array
+    bad_off = b["key_off"].copy()
+    bad_off[1] += 2
+    bad_off[3] = -8
+    idx, cnt, kth = B.janus_topk_batch(good, torch.from_numpy(bad_off).cuda(), k, row_lengths=row_len)
+    assert _status_word() == 101
+    idx_h, cnt_h = idx.cpu().numpy(), cnt.cpu().numpy()
+    assert (idx_h[1] == -1).all() and (idx_h[3] == -1).all() and cnt_h[1] == 0 and cnt_h[3] == 0
+    assert np.isneginf(kth.cpu().numpy()[[1, 3]]).all()
+    for i in (0, 2):
+        assert set(idx_h[i].tolist()) == set(idx_good[i].cpu().numpy().tolist()) and cnt_h[i] == int(cnt_good[i])
+    # a negative length
+    bad_len = row_len.clone()
+    bad_len[2] = -5
+    idx, cnt, _ = B.janus_topk_batch(good, key_off, k, row_lengths=bad_len)
+    assert _status_word() == 101 and int(cnt[2]) == 0 and (idx[2] == -1).all()
+
+    # ---- janus_indexer_scores_batch: the last session claims rows beyond the key array, session 1 starts before it
+    canary = torch.full((total + 4096,), 7.5, dtype=torch.float32, device="cuda")
+    over = b["key_off"].copy()
+    over[-1] = total + 3000
+    sc = B.janus_indexer_scores_batch(qd, kd, wd, torch.from_numpy(over).cuda(), max(lengths) + 4, q_scale=qs, k_scale=ks, scores=canary[:total])
+    assert _status_word() == 101
+    assert (canary[total:] == 7.5).all()                       # nothing was written past the score array
+    a0, a3 = int(b["key_off"][0]), int(b["key_off"][3])
+    assert torch.equal(sc[a0:a0 + lengths[0] + 1], good[a0:a0 + lengths[0] + 1])
+    assert torch.equal(sc[a3:total], good[a3:total])           # the part of the cut session that lies inside the array
+    neg = b["key_off"].copy()
+    neg[1] = -4
+    sc = B.janus_indexer_scores_batch(qd, kd, wd, torch.from_numpy(neg).cuda(), max(lengths) + 4, q_scale=qs, k_scale=ks)
+    assert _status_word() == 101
+    a2 = int(b["key_off"][2])
+    assert torch.equal(sc[a2:a2 + lengths[2] + 1], good[a2:a2 + lengths[2] + 1])
+
+    # ---- janus_page_demand_batch: a negative page-table offset empties that row's table
+    tab_off = torch.from_numpy(b["tab_off"]).cuda()
+    limits = torch.tensor(lengths, dtype=torch.int64, device="cuda")
+    tables = dev(b["tables"], "i32")
+    neg_tab = b["tab_off"].copy()
+    neg_tab[2] = -3
+    pd = B.janus_page_demand_batch(idx_good, demand_limits=limits, page_size=page, page_tables=tables, table_offsets=torch.from_numpy(neg_tab).cuda(),
+                                   n_phys_pages=b["n_phys"])
+    assert _status_word() == 101
+    idx_gh = idx_good.cpu().numpy()
+    want = set()
+    for i, L in enumerate(lengths):
+        if i in (1, 2):      # row 1's table now ends at a negative offset (length < 0), row 2's starts at one: both are empty
+            continue
+        want |= set(O.page_demand(idx_gh[i:i + 1], L, page, b["tables"][b["tab_off"][i]:b["tab_off"][i + 1]])["pages"])
+    assert Hp.page_lists_from_device(pd)["pages"] == sorted(want)
+
+    # ---- janus_sparse_attn_decode: a negative physical page id is skipped like a padding slot
+    rng = np.random.default_rng(9)
+    q_attn = W.to_bf16_bits((rng.standard_normal((nb, H_q, d_qk)) / 4).astype(np.float32))
+    pool = W.to_bf16_bits((rng.standard_normal((b["n_phys"], page, 1, d_qk)) / 4).astype(np.float32))
+    bad_tables = b["tables"].copy()
+    lp_bad = 3                                                   # session 0, logical page 3
+    bad_tables[b["tab_off"][0] + lp_bad] = -1
+    pool_d = dev(pool, "bf16")
+    scale = 1.0 / np.sqrt(d_qk)
+    out, _ = B.janus_sparse_attn_decode(dev(q_attn, "bf16"), pool_d, pool_d, idx_good, page_tables=dev(bad_tables, "i32"), table_offsets=tab_off,
+                                        page_size=page, softmax_scale=scale, d_v=d_v)
+    hit = (idx_gh[0] >= 0) & (idx_gh[0] // page == lp_bad)
+    st = _status_word()
+    assert st == (101 if hit.any() else 0)
+    idx_ref = idx_gh[0:1].copy()
+    idx_ref[0, hit] = -1                                         # the oracle on the selection without the skipped tokens
+    ref_o, _ = O.sparse_attention(q_attn[0:1], pool, pool, b["tables"][b["tab_off"][0]:b["tab_off"][1]], idx_ref, page_size=page,
+                                  softmax_scale=scale, d_qk=d_qk, d_v=d_v)
+    Hp.assert_attention_close(Hp.bf16_tensor_to_f64(out)[0:1], ref_o, "attention with a negative page id")
+
+    # an ordinary call afterwards is clean
+    again = B.janus_indexer_scores_batch(qd, kd, wd, key_off, max(lengths) + 4, q_scale=qs, k_scale=ks)
+    B.check_dev_status()
+    assert torch.equal(again, good)
