@@ -94,6 +94,53 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def probe_fp8_peak(seconds: float = 1.0):
+    """Dense FP8 tensor rate of this GPU, measured outside the timed region (TFLOP/s): the library's own tcgen05 loop
+    (operands in shared memory, M = 128, N = 256, the indexer's instruction shape) and, as a library cross-check, a
+    torch._scaled_mm E4M3 GEMM of 8192^3.  `burst` = best of several short launches; `sustained` = back to back for about
+    `seconds` (the rate the power limit allows, which is what a kernel inside a long step sees)."""
+    import torch
+    from paper_2609_36938_b200 import binding as B
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    out = {}
+    n_sm = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+
+    def timed(fn, flop, reps):
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return flop * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12, e0.elapsed_time(e1) * 1e-3
+
+    fills = 4096                                             # 5.1 TFLOP per launch, under 2 ms
+    flop = 2.0 * 128 * 256 * 128 * fills * n_sm
+    own = lambda: B.janus_fp8_mma_probe(n_sm, fills)
+    own(); torch.cuda.synchronize()
+    out["own_loop_burst"] = max(timed(own, flop, 1)[0] for _ in range(10))
+    rate, dt = timed(own, flop, 50)
+    reps = max(50, int(50 * seconds / dt))
+    out["own_loop_sustained"] = timed(own, flop, reps)[0]
+    B.check_dev_status()
+    try:
+        n = 8192
+        a = torch.randn((n, n), device="cuda").to(torch.float8_e4m3fn)
+        b = torch.randn((n, n), device="cuda").to(torch.float8_e4m3fn).t()     # column-major second operand
+        one = torch.ones((), device="cuda")
+        mm = lambda: torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+        mm(); torch.cuda.synchronize()
+        gflop = 2.0 * n * n * n
+        out["scaled_mm_burst"] = max(timed(mm, gflop, 1)[0] for _ in range(10))
+        rate, dt = timed(mm, gflop, 50)
+        out["scaled_mm_sustained"] = timed(mm, gflop, max(50, int(50 * seconds / dt)))[0]
+        del a, b
+    except Exception as e:      # the probe is a cross-check only
+        out["scaled_mm_error"] = f"{type(e).__name__}: {e}"[:200]
+    return {k: (round(v, 1) if isinstance(v, float) else v) for k, v in out.items()}
+
+
 def captured_traffic(kernel_key: str, rows: int):
     """DRAM bytes of one launch of `kernel_key`, from the ncu capture summarised under profiles/ (a small case of the same
     kernel), scaled by query rows to this launch.  None if no capture is recorded."""
@@ -236,13 +283,102 @@ def run_decode(args):
     print(json.dumps(line))
 
 
+def run_sharded_prediction(args, rank, world, local_rank):
+    """--shard keys: the synchronisation-free parallel prediction of Sec. 4.2 (Eq. 3) across ranks.  Every rank holds the
+    lookahead queries and its own disjoint, page-aligned shard C_n of the history keys; a step is indexer -> top-(k/N) ->
+    page demand on that shard (no exchange: the rank could start prefetching its pages here) followed by the one
+    exchange of the partition, the union of the ranks' page bitmaps that the exact pass is compared against.  The whole
+    job's work is fixed (one session's prediction pass), so scaling is strong.  The session is the first one of the
+    ragged batch (config 4), the configuration whose predicted set is defined."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_36938_b200 import binding as B, build as _build, dist_utils as D, prediction as P, report as R, workloads as W
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    B.load()
+    shp = W.batch_shapes(args.seed)[0] if (args.L is None and args.M is None) else W.config_shape(4, L=args.L, M=args.M)
+    sess = W.make_session(shp, args.seed, with_attention=False, page_table=W.make_page_table(
+        W.config_shape(2, L=shp.L, M=shp.M), args.seed), n_phys_pages=shp.n_logical_pages)
+    n_phys = sess["n_phys_pages"]
+    kind = shp.idx_dtype
+    bounds = P.shard_bounds(shp.L, world, shp.page_size)
+    a, b = bounds[rank] if rank < len(bounds) else (0, 0)
+    k_shard = max(1, shp.k // world)
+    q_pred = B.to_device(sess["q_pred"], kind)
+    w = B.to_device(sess["w"], "f32")
+    k_mine = B.to_device(sess["k_idx"][a:b], kind)
+    table = B.to_device(sess["page_table"], "i32")
+    table_mine = table[a // shp.page_size:]
+    ld = ((b - a) + 31) // 32 * 32
+    scores = torch.empty((shp.M, max(ld, 32)), dtype=torch.float32, device="cuda")
+    idx = torch.empty((shp.M, k_shard), dtype=torch.int32, device="cuda")
+    bufs = B.page_demand_buffers(n_phys, want_miss=False)
+    union_fn = lambda dst, src: B.janus_page_union(dst, src, n_phys)
+
+    def step():
+        sc = B.janus_indexer_scores(q_pred, k_mine, w, q_pos0=shp.L, causal=False, scores=scores)
+        B.janus_topk(sc, b - a, k_shard, q_pos0=shp.L, causal=False, want_count=False, want_kth=False, idx=idx)
+        pd = B.janus_page_demand(idx, demand_limit=b - a, page_size=shp.page_size, page_table=table_mine, n_phys_pages=n_phys, want_miss=False, out=bufs)
+        return D.or_reduce_bitmap(pd["bitmap"], union_fn)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        sampler.wait_until_running()
+    for _ in range(max(args.warmup, 3)):
+        union = step()
+    B.check_dev_status()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        union = step()
+    e1.record()
+    barrier()
+    B.check_dev_status()
+    # strong scaling: every rank reports the whole session's M tokens once (rank 0 only), the time is the maximum over ranks
+    value, elapsed_ms, _ = D.aggregate_throughput(float(shp.M * args.steps) if rank == 0 else 0.0, e0.elapsed_time(e1), device="cuda")
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        # untimed: the exact pass of the same session on this rank, and what the united prediction covers of it
+        k_all = B.to_device(sess["k_idx"], kind)
+        sc = B.janus_indexer_scores(B.to_device(sess["q_idx"], kind), k_all, w, q_pos0=shp.L, causal=True)
+        eidx, _, _ = B.janus_topk(sc, shp.S, shp.k, q_pos0=shp.L, causal=True, want_count=False, want_kth=False)
+        pd = B.janus_page_demand(eidx, demand_limit=shp.L, page_size=shp.page_size, page_table=table, n_phys_pages=n_phys, predicted_bitmap=union)
+        rep = R.demand_report(pd, union)
+        B.check_dev_status()
+        line = {"metric": "sharded_prediction_new_tokens_per_sec_per_sparse_layer", "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                "dtype": kind, "data": "synthetic", "clocks": clocks,
+                "config": {"workload": f"key-sharded prediction pass (Eq. 3): L={shp.L} M={shp.M} k={shp.k} -> top-{k_shard} per shard, {world} page-aligned "
+                                       f"history shards, indexer {shp.H_I}x{shp.D_I} {kind}, page {shp.page_size}, shuffled page table",
+                           "exchange": "one all-gather of the page bitmaps + local union (janus_page_union) per step"},
+                "gpu_launches": 5 * args.steps, "page_report_vs_exact": rep}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, help="benchmark configuration 1..5 (4 = first session of the ragged batch)")
+    ap.add_argument("--workload", type=int, default=3, help="benchmark configuration 1..5 (4 = the ragged batch of 8 sessions, one after another)")
+    ap.add_argument("--sessions", type=int, default=None, help="with --workload 4: only the first N sessions of the batch")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--L", type=int, default=None)
     ap.add_argument("--M", type=int, default=None)
@@ -250,6 +386,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the side measurement of janus_indexer_topk")
+    ap.add_argument("--no-peak-probe", action="store_true", help="skip the FP8 tensor-rate probe (the roofline then divides by an assumed peak)")
+    ap.add_argument("--no-report", action="store_true", help="skip the recall / precision / run-length report of configs 1, 4, 5")
+    ap.add_argument("--shard", default="none", choices=["none", "keys"],
+                    help="keys: with --gpus N, time the key-sharded prediction pass (Eq. 3): rank n scores its own history shard")
     ap.add_argument("--decode-batch", type=int, default=0, help="side workload: time one decode step over this many sessions instead")
     ap.add_argument("--decode-fp4-keys", action="store_true", help="with --decode-batch: indexer keys stored as FP4 E2M1")
     args = ap.parse_args()
@@ -263,22 +403,40 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.shard == "keys" and args.impl == "ours":
+        run_sharded_prediction(args, rank, world, local_rank)
+        return
 
     from paper_2609_36938_b200 import workloads as W
 
-    if args.workload == 4:
-        shp = W.batch_shapes(args.seed)[0]
+    if args.workload == 4 and args.L is None and args.M is None:
+        shapes = W.batch_shapes(args.seed)
+        if args.sessions:
+            shapes = shapes[:args.sessions]
     else:
-        shp = W.config_shape(args.workload, L=args.L, M=args.M)
-    workload_name = (f"config {args.workload}: L={shp.L} M={shp.M} k={shp.k}, indexer {shp.H_I}x{shp.D_I} {shp.idx_dtype}, "
+        shapes = [W.config_shape(args.workload, L=args.L, M=args.M)]
+    n_sessions = len(shapes)
+    shp = shapes[0]
+    if n_sessions == 1:
+        sizes = f"L={shp.L} M={shp.M}"
+    else:
+        sizes = f"{n_sessions} sessions one after another, L={[x.L for x in shapes]} M={[x.M for x in shapes]}"
+    workload_name = (f"config {args.workload}: {sizes} k={shp.k}, indexer {shp.H_I}x{shp.D_I} {shp.idx_dtype}, "
                      f"{shp.attn} attention {shp.H_q} heads {shp.d_qk}/{shp.d_v} bf16, page {shp.page_size}, {shp.table} page table")
-    config = {"workload": workload_name, "sessions_per_gpu": 1, "cache": "inputs larger than L2 (scores, Q and gathered KV are GBs per step)"}
+    config = {"workload": workload_name, "sessions_per_gpu": n_sessions, "cache": "inputs larger than L2 (scores, Q and gathered KV are GBs per step)"}
+
+    def make_sessions(seed):
+        if n_sessions > 1 or shp.table == "fragmented":
+            return W.make_batch(seed, shapes)
+        return [W.make_session(shp, seed)]
 
     if args.impl == "reference":
         if rank != 0:
             return
-        sess = W.make_session(shp, args.seed)
+        sess = make_sessions(args.seed)[0]
         cb = run_reference(args, shp, sess)
+        if n_sessions > 1:
+            cb["sample"] = "first session of the batch: " + cb["sample"]
         line = {"metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps_ref, "warmup": args.warmup_ref,
                 "ms_per_step": cb["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
                 "data": "synthetic", "config": config, "impl": "reference",
@@ -290,7 +448,7 @@ def main():
     import torch
     import torch.distributed as dist
 
-    from paper_2609_36938_b200 import binding as B, build as _build, dist_utils as D
+    from paper_2609_36938_b200 import binding as B, build as _build, dist_utils as D, report as R
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -303,69 +461,100 @@ def main():
         dist.barrier()
     B.load()
 
-    sess = W.make_session(shp, args.seed + rank)
+    sessions = make_sessions(args.seed + rank)
     kind = shp.idx_dtype
-    host = {
-        "q_idx": (sess["q_idx"], kind), "k_idx": (sess["k_idx"], kind), "w": (sess["w"], "f32"), "q_scale": (sess["q_scale"], "f32"),
-        "k_scale": (sess["k_scale"], "f32"), "row_bias": (sess["row_bias"], "f32"), "col_bias": (sess["col_bias"], "f32"),
-        "page_table": (sess["page_table"], "i32"), "Q": (sess["Q"], "bf16"), "k_pool": (sess["k_pool"], "bf16"),
-    }
-    if sess["v_pool"] is not sess["k_pool"]:
-        host["v_pool"] = (sess["v_pool"], "bf16")
-    pinned = {}
-    for name, (arr, kd) in host.items():
+    tokens_per_step = sum(x.M for x in shapes)
+    n_phys = sessions[0]["n_phys_pages"]
+
+    # pinned host copies of every operand; tensors shared by sessions (the KV pool of a batch) are held, uploaded and counted once
+    pinned_by_id = {}
+
+    def pin(arr, kd):
         if arr is None:
-            pinned[name] = None
+            return None
+        if id(arr) not in pinned_by_id:
+            pinned_by_id[id(arr)] = B.to_device(arr, kd, device="cpu").pin_memory()
+        return pinned_by_id[id(arr)]
+
+    pinned = []
+    for sess in sessions:
+        pinned.append({
+            "q_idx": pin(sess["q_idx"], kind), "k_idx": pin(sess["k_idx"], kind), "w": pin(sess["w"], "f32"), "q_scale": pin(sess["q_scale"], "f32"),
+            "k_scale": pin(sess["k_scale"], "f32"), "row_bias": pin(sess["row_bias"], "f32"), "col_bias": pin(sess["col_bias"], "f32"),
+            "page_table": pin(sess["page_table"], "i32"), "Q": pin(sess["Q"], "bf16"), "k_pool": pin(sess["k_pool"], "bf16"),
+            "v_pool": pin(sess["v_pool"], "bf16"),
+        })
+    h2d_bytes = sum(t.numel() * t.element_size() for t in pinned_by_id.values())
+
+    def device_set():
+        """One device copy of every distinct pinned tensor, and the per-session views onto them."""
+        dev_by_id = {i: torch.empty_like(t, device="cuda") for i, t in pinned_by_id.items()}
+        by_pin = {id(t): dev_by_id[i] for i, t in pinned_by_id.items()}
+        views = [{n: (None if t is None else by_pin[id(t)]) for n, t in pn.items()} for pn in pinned]
+        return dev_by_id, views
+
+    def upload_all(dev_by_id):
+        for i, t in pinned_by_id.items():
+            dev_by_id[i].copy_(t, non_blocking=True)
+
+    dev0, d_list = device_set()
+    upload_all(dev0)
+    ld_max = max((x.S + 31) // 32 * 32 for x in shapes)
+    scores_buf = torch.empty((max(x.M for x in shapes) * ld_max,), dtype=torch.float32, device="cuda")
+    out_bufs = [torch.empty((x.M, x.H_q, x.d_v), dtype=torch.bfloat16, device="cuda") for x in shapes]
+    idx_bufs = [torch.empty((x.M, x.k), dtype=torch.int32, device="cuda") for x in shapes]
+
+    def scores_view(x):
+        ld = (x.S + 31) // 32 * 32
+        return scores_buf[:x.M * ld].view(x.M, ld)
+
+    # predicted pass (Eq. 2): same indexer on the lookahead queries over the history keys only; prepared once per session
+    pred_bitmaps, pred_idx = [], []
+    for x, sess, d in zip(shapes, sessions, d_list):
+        if "q_pred" not in sess:
+            pred_bitmaps.append(None); pred_idx.append(None)
             continue
-        t = B.to_device(arr, kd, device="cpu")
-        pinned[name] = t.pin_memory()
-    h2d_bytes = sum(t.numel() * t.element_size() for t in pinned.values() if t is not None)
-
-    def upload():
-        d = {n: (None if t is None else t.to("cuda", non_blocking=True)) for n, t in pinned.items()}
-        if "v_pool" not in d:
-            d["v_pool"] = d["k_pool"]
-        return d
-
-    d = upload()
-    n_phys = sess["n_phys_pages"]
-    ld = (shp.S + 31) // 32 * 32
-    scores = torch.empty((shp.M, ld), dtype=torch.float32, device="cuda")
-    out_buf = torch.empty((shp.M, shp.H_q, shp.d_v), dtype=torch.bfloat16, device="cuda")
-
-    # predicted pass (Eq. 2): same indexer on the lookahead queries over the history keys only; prepared once
-    pred_bitmap = None
-    if "q_pred" in sess:
         qp = B.to_device(sess["q_pred"], kind)
-        psc = B.janus_indexer_scores(qp, d["k_idx"][:shp.L], d["w"], q_scale=d["q_scale"],
-                                     k_scale=None if d["k_scale"] is None else d["k_scale"][:shp.L], q_pos0=shp.L, causal=False)
-        pidx, _, _ = B.janus_topk(psc, shp.L, shp.k, q_pos0=shp.L, causal=False, want_count=False, want_kth=False)
-        pred_bitmap = B.janus_page_demand(pidx, demand_limit=shp.L, page_size=shp.page_size, page_table=d["page_table"],
-                                          n_phys_pages=n_phys, want_miss=False)["bitmap"]
-        del psc, pidx, qp
+        psc = B.janus_indexer_scores(qp, d["k_idx"][:x.L], d["w"], q_scale=d["q_scale"],
+                                     k_scale=None if d["k_scale"] is None else d["k_scale"][:x.L], q_pos0=x.L, causal=False)
+        pidx, _, _ = B.janus_topk(psc, x.L, x.k, q_pos0=x.L, causal=False, want_count=False, want_kth=False)
+        pred_bitmaps.append(B.janus_page_demand(pidx, demand_limit=x.L, page_size=x.page_size, page_table=d["page_table"],
+                                                n_phys_pages=n_phys, want_miss=False)["bitmap"])
+        pred_idx.append(pidx)
+        del psc, qp
+    torch.cuda.empty_cache()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     stream = torch.cuda.current_stream()
+    pd_bufs = [B.page_demand_buffers(n_phys) for _ in shapes]      # allocated once: the timed path neither allocates nor fills
 
-    def step(d, marks=None, out_to=None):
+    def session_step(b, d, marks=None, out_to=None):
+        """The four calls of the exact pass of session b on the device operands d."""
+        x = shapes[b]
         if marks is not None:
             marks[0].record(stream)
         sc = B.janus_indexer_scores(d["q_idx"], d["k_idx"], d["w"], q_scale=d["q_scale"], k_scale=d["k_scale"], row_bias=d["row_bias"],
-                                    col_bias=d["col_bias"], q_pos0=shp.L, causal=True, scores=scores)
+                                    col_bias=d["col_bias"], q_pos0=x.L, causal=True, scores=scores_view(x))
         if marks is not None:
             marks[1].record(stream)
-        idx, _, _ = B.janus_topk(sc, shp.S, shp.k, q_pos0=shp.L, causal=True, want_count=False, want_kth=False)
+        idx, _, _ = B.janus_topk(sc, x.S, x.k, q_pos0=x.L, causal=True, want_count=False, want_kth=False, idx=idx_bufs[b])
         if marks is not None:
             marks[2].record(stream)
-        pd = B.janus_page_demand(idx, demand_limit=shp.L, page_size=shp.page_size, page_table=d["page_table"], n_phys_pages=n_phys,
-                                 predicted_bitmap=pred_bitmap)
+        pd = B.janus_page_demand(idx, demand_limit=x.L, page_size=x.page_size, page_table=d["page_table"], n_phys_pages=n_phys,
+                                 predicted_bitmap=pred_bitmaps[b], out=pd_bufs[b])
         if marks is not None:
             marks[3].record(stream)
-        out, _ = B.janus_sparse_attn_prefill(d["Q"], d["k_pool"], d["v_pool"], idx, page_table=d["page_table"], page_size=shp.page_size,
-                                             softmax_scale=shp.softmax_scale, d_v=shp.d_v, want_lse=False, out=out_buf if out_to is None else out_to)
+        out, _ = B.janus_sparse_attn_prefill(d["Q"], d["k_pool"], d["v_pool"], idx, page_table=d["page_table"], page_size=x.page_size,
+                                             softmax_scale=x.softmax_scale, d_v=x.d_v, want_lse=False, out=out_bufs[b] if out_to is None else out_to)
         if marks is not None:
             marks[4].record(stream)
         return idx, pd, out
+
+    def step(marks=None):
+        res = None
+        for b in range(n_sessions):
+            res = session_step(b, d_list[b], None if marks is None else marks[b])
+        return res
 
     def barrier():
         if world > 1:
@@ -379,71 +568,67 @@ def main():
     if world > 1:
         dist.barrier()
     for _ in range(args.warmup):
-        step(d)
+        step()
     B.check_dev_status()
 
     # ---- timed region: device-resident inputs
-    marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    marks = [[[ev() for _ in range(5)] for _ in range(n_sessions)] for _ in range(args.steps)]
     barrier()
     t_start, t_end = ev(), ev()
     t_start.record(stream)
     for i in range(args.steps):
-        idx, pd, out = step(d, marks[i])
+        idx, pd, out = step(marks[i])
     t_end.record(stream)
     barrier()
     B.check_dev_status()
     elapsed_ms = t_start.elapsed_time(t_end)
-    per_call = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])   # [steps, 4] ms
-    value, elapsed_ms, _ = D.aggregate_throughput(float(shp.M * args.steps), elapsed_ms, device="cuda")   # max over ranks
+    # [steps, 4] ms: per call, summed over the sessions of a step
+    per_call = np.array([[sum(m[b][j].elapsed_time(m[b][j + 1]) for b in range(n_sessions)) for j in range(4)] for m in marks])
+    per_session_ms = [float(np.mean([m[b][0].elapsed_time(m[b][4]) for m in marks])) for b in range(n_sessions)]
+    value, elapsed_ms, _ = D.aggregate_throughput(float(tokens_per_step * args.steps), elapsed_ms, device="cuda")   # max over ranks
     ms_per_step = elapsed_ms / args.steps
 
     # ---- end to end: every step uploads all inputs from pinned host memory and reads the results back
     e2e = None
     if not args.no_e2e:
-        host_out = torch.empty(out_buf.shape, dtype=out_buf.dtype).pin_memory()
-        host_idx = torch.empty((shp.M, shp.k), dtype=torch.int32).pin_memory()
+        host_out = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in out_bufs]
+        host_idx = [torch.empty(ib.shape, dtype=torch.int32).pin_memory() for ib in idx_bufs]
         host_pages = torch.empty((n_phys,), dtype=torch.int32).pin_memory()
         host_counts = torch.empty((4,), dtype=torch.int32).pin_memory()
-        d2h_bytes = sum(t.numel() * t.element_size() for t in (host_out, host_idx, host_pages, host_counts))
+        d2h_bytes = sum(t.numel() * t.element_size() for t in host_out + host_idx) + n_sessions * (host_pages.numel() + 4) * 4
 
         # Three streams, two sets of device buffers: the upload of step i+1 and the read-back of step i-1 run while step i
         # computes, as a serving loop would do it.  Every step still copies all of its inputs from pinned host memory and
         # all of its results back; the timed region covers all of it.
         s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-        dev_in = [{n: (None if t is None else torch.empty_like(t, device="cuda")) for n, t in pinned.items()} for _ in range(2)]
-        for dd in dev_in:
-            if "v_pool" not in dd:
-                dd["v_pool"] = dd["k_pool"]
-        dev_out = [torch.empty_like(out_buf) for _ in range(2)]
+        dev_sets = [device_set() for _ in range(2)]
+        dev_out = [[torch.empty_like(o) for o in out_bufs] for _ in range(2)]
         in_done = [ev() for _ in range(2)]
         cmp_done = [ev() for _ in range(2)]
         out_done = [ev() for _ in range(2)]
 
         def e2e_steps(n):
             for i in range(n):
-                b = i & 1
+                s2 = i & 1
                 with torch.cuda.stream(s_in):
                     if i >= 2:
-                        s_in.wait_event(cmp_done[b])          # step i-2 has finished reading this input set
-                    for name, t in pinned.items():
-                        if t is not None:
-                            dev_in[b][name].copy_(t, non_blocking=True)
-                    in_done[b].record(s_in)
+                        s_in.wait_event(cmp_done[s2])          # step i-2 has finished reading this input set
+                    upload_all(dev_sets[s2][0])
+                    in_done[s2].record(s_in)
                 with torch.cuda.stream(s_cmp):
-                    s_cmp.wait_event(in_done[b])
+                    s_cmp.wait_event(in_done[s2])
                     if i >= 2:
-                        s_cmp.wait_event(out_done[b])         # step i-2's output buffer has been read back
-                    idx, pd, out = step(dev_in[b], out_to=dev_out[b])
-                    cmp_done[b].record(s_cmp)
+                        s_cmp.wait_event(out_done[s2])         # step i-2's output buffers have been read back
+                    results = [session_step(b, dev_sets[s2][1][b], out_to=dev_out[s2][b]) for b in range(n_sessions)]
+                    cmp_done[s2].record(s_cmp)
                 with torch.cuda.stream(s_out):
-                    s_out.wait_event(cmp_done[b])
-                    for t in (idx, pd["pages"], pd["counts"]):
-                        t.record_stream(s_out)
-                    host_out.copy_(out, non_blocking=True)
-                    host_idx.copy_(idx, non_blocking=True)
-                    host_pages.copy_(pd["pages"][:n_phys], non_blocking=True)
-                    host_counts.copy_(pd["counts"], non_blocking=True)
-                    out_done[b].record(s_out)
+                    s_out.wait_event(cmp_done[s2])
+                    for b, (ridx, rpd, rout) in enumerate(results):
+                        host_out[b].copy_(rout, non_blocking=True)
+                        host_idx[b].copy_(ridx, non_blocking=True)
+                        host_pages.copy_(rpd["pages"][:n_phys], non_blocking=True)
+                        host_counts.copy_(rpd["counts"], non_blocking=True)
+                    out_done[s2].record(s_out)
             for st in (s_in, s_cmp, s_out):
                 stream.wait_stream(st)
 
@@ -457,24 +642,51 @@ def main():
         e2e_steps(n_e2e)
         e1.record(stream)
         barrier()
-        e2e_value, e2e_total_ms, _ = D.aggregate_throughput(float(shp.M * n_e2e), e0.elapsed_time(e1), device="cuda")
+        e2e_value, e2e_total_ms, _ = D.aggregate_throughput(float(tokens_per_step * n_e2e), e0.elapsed_time(e1), device="cuda")
         e2e_ms = e2e_total_ms / n_e2e
         e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(d2h_bytes),
                "ms_per_step": e2e_ms, "inputs": "all operands (queries, keys, weights, Q, KV pool, page table) uploaded every step; upload, compute and read-back of "
                          "consecutive steps overlap on three streams (two buffer sets)"}
+        del dev_sets, dev_out
+        torch.cuda.empty_cache()
 
     # a short run can end between two samples: keep the same load on until one sample has been taken under it
     if rank == 0 and sampler.proc is not None:
         t_wait = time.time()
         while len(sampler.rows) - sampler.skip < 2 and time.time() - t_wait < 2.0:
-            step(d)
+            step()
             torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- report (untimed, from the device outputs of the last step): recall / precision of the predicted page set against the
+    # exact one, miss-set size, runs, the same at token granularity, and the run-length histogram (shuffled and identity table)
+    report = None
+    if rank == 0 and not args.no_report and (args.workload in (1, 4, 5)):
+        report = {"sessions": []}
+        for b, x in enumerate(shapes):
+            r = {"L": x.L, "M": x.M, "pages": R.demand_report(pd_bufs[b], pred_bitmaps[b]),
+                 "tokens": R.token_granularity_report(idx_bufs[b], pred_idx[b], x.L)}
+            if args.workload == 5 or n_sessions == 1:
+                r["run_length_histogram"] = {str(k_): v for k_, v in sorted(R.run_length_histogram(pd_bufs[b]).items())}
+                ident = torch.arange(x.n_logical_pages, dtype=torch.int32, device="cuda")
+                pd_id = B.janus_page_demand(idx_bufs[b], demand_limit=x.L, page_size=x.page_size, page_table=ident, n_phys_pages=x.n_logical_pages, want_miss=False)
+                r["identity_table"] = {"n_runs": int(pd_id["counts"][1].item()), "n_pages": int(pd_id["counts"][0].item()),
+                                       "run_length_histogram": {str(k_): v for k_, v in sorted(R.run_length_histogram(pd_id).items())}}
+            report["sessions"].append(r)
+        if any(p_ is not None for p_ in pred_bitmaps):
+            for level in ("pages", "tokens"):
+                report[f"mean_{level}_recall"] = float(np.mean([r[level]["recall"] for r in report["sessions"]]))
+                report[f"mean_{level}_precision"] = float(np.mean([r[level]["precision"] for r in report["sessions"]]))
+                report[f"mean_{level}_miss"] = float(np.mean([r[level]["n_miss"] for r in report["sessions"]]))
+        B.check_dev_status()
+
     # ---- side measurement (not part of `value`): indexer + top-k as one call that never stores the score matrix
     fused = None
-    if not args.no_fused:
+    if not args.no_fused and n_sessions == 1:
         lib = B.load()
+        d = d_list[0]
         ws_bytes = int(lib.janus_indexer_topk_workspace_size(shp.M, shp.H_I, shp.D_I, shp.S, shp.L, 1, 1 if shp.idx_dtype == "fp8" else 0, shp.k))
-        del scores
+        del scores_buf
         torch.cuda.empty_cache()
         ws = torch.empty((ws_bytes,), dtype=torch.uint8, device="cuda")
         fidx = torch.empty((shp.M, shp.k), dtype=torch.int32, device="cuda")
@@ -494,20 +706,41 @@ def main():
         barrier()
         B.check_dev_status()
         fused = {"ms": f0.elapsed_time(f1) / 5, "two_call_ms": float(per_call[:, 0].mean() + per_call[:, 1].mean()), "workspace_bytes": ws_bytes,
-                 "score_matrix_bytes": int(shp.M) * int(ld) * 4}
+                 "score_matrix_bytes": int(shp.M) * int((shp.S + 31) // 32 * 32) * 4,
+                 "note": "one call that never stores the score matrix: a memory-saving path (workspace vs score matrix), not the faster one at this size"}
 
-    clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     peaks = load_peaks()
-    wn = workload_numbers(shp)
+    wns = [workload_numbers(x) for x in shapes]
+    wn = {k_: sum(w_[k_] for w_ in wns) for k_ in wns[0]}
     mean_ms = per_call.mean(axis=0)
     names = ["indexer_scores", "topk", "page_demand", "sparse_attn_prefill"]
     fp8 = shp.idx_dtype == "fp8"
-    tensor_peak_idx = peaks["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)
+    # FP8 tensor peak: measured in this run (sustained: the indexer runs inside a long step); the larger of the library's own
+    # tcgen05 loop and the torch._scaled_mm GEMM, so that the fraction is never flattered.  Twice the measured bf16 figure
+    # (the nominal ratio) is kept beside it.
+    fp8_probe = None
+    assumed_fp8 = peaks["bf16_tflops_sustained"] * 2.0
+    if fp8 and not args.no_peak_probe:
+        fp8_probe = probe_fp8_peak()
+        fp8_probe["assumed_2x_bf16_sustained"] = assumed_fp8
+    if fp8:
+        if fp8_probe is not None:
+            tensor_peak_idx = max(fp8_probe.get("own_loop_sustained", 0.0), fp8_probe.get("scaled_mm_sustained", 0.0))
+            peak_source_idx = ("measured in this run: sustained dense FP8 E4M3 rate, max of the library's own tcgen05 loop "
+                               f"({fp8_probe.get('own_loop_sustained')} TFLOP/s) and torch._scaled_mm 8192^3 ({fp8_probe.get('scaled_mm_sustained')} TFLOP/s)")
+        else:
+            tensor_peak_idx = assumed_fp8
+            peak_source_idx = f"ASSUMED: {peaks['source']} bf16 sustained x2 (nominal fp8:bf16 ratio); no FP8 probe in this run"
+    else:
+        tensor_peak_idx = peaks["bf16_tflops_sustained"]
+        peak_source_idx = f"{peaks['source']} bf16 sustained"
+    rows_total = sum(x.M for x in shapes)
+    attn_dram = captured_traffic("sparse_attn_latent", rows_total) if shp.attn == "latent" else None
     kernels = {
         "indexer_scores": {"ms": mean_ms[0], "tflops": wn["indexer_flops"] / (mean_ms[0] * 1e-3) / 1e12,
                            "frac_tensor_peak": wn["indexer_flops"] / (mean_ms[0] * 1e-3) / 1e12 / tensor_peak_idx},
@@ -516,40 +749,56 @@ def main():
         "page_demand": {"ms": mean_ms[2], "gbs": wn["page_demand_bytes"] / (mean_ms[2] * 1e-3) / 1e9},
         "sparse_attn_prefill": {"ms": mean_ms[3], "tflops": wn["attn_flops"] / (mean_ms[3] * 1e-3) / 1e12,
                                 "logical_gbs": wn["attn_bytes"] / (mean_ms[3] * 1e-3) / 1e9,
-                                "frac_hbm_peak": wn["attn_bytes"] / (mean_ms[3] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "frac_hbm_peak_logical": wn["attn_bytes"] / (mean_ms[3] * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                 "frac_tensor_peak": wn["attn_flops"] / (mean_ms[3] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
     }
+    if attn_dram is not None:    # what actually came from DRAM (ncu capture, scaled by rows): most gathered rows are L2 hits
+        kernels["sparse_attn_prefill"]["dram_gbs_captured"] = attn_dram / (mean_ms[3] * 1e-3) / 1e9
+        kernels["sparse_attn_prefill"]["frac_hbm_peak_dram"] = attn_dram / (mean_ms[3] * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    kernels["topk_plus_gather"] = {"ms": mean_ms[1] + mean_ms[3], "logical_gbs": (wn["topk_bytes"] + wn["attn_bytes"]) / ((mean_ms[1] + mean_ms[3]) * 1e-3) / 1e9,
+                                   "frac_hbm_peak_logical": (wn["topk_bytes"] + wn["attn_bytes"]) / ((mean_ms[1] + mean_ms[3]) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     dom = int(np.argmax(mean_ms))
     if names[dom] == "indexer_scores":
         roofline = {"kernel": "indexer_tc_kernel", "bound": "tensor", "achieved": kernels["indexer_scores"]["tflops"], "peak": tensor_peak_idx,
                     "unit": "TFLOP/s", "frac": kernels["indexer_scores"]["frac_tensor_peak"],
-                    "traffic": captured_traffic("indexer_tc" if fp8 else "indexer_tc_bf16", shp.M),
-                    "traffic_note": "ncu dram bytes of a 296-row capture of the same kernel scaled by rows (profiles/); for bf16 the capture is at L=32768",
-                    "peak_source": f"{peaks['source']} bf16 sustained" + (" x2 (nominal fp8:bf16 ratio)" if fp8 else "")}
+                    "traffic": captured_traffic("indexer_tc" if fp8 else "indexer_tc_bf16", rows_total),
+                    "traffic_note": "ncu dram bytes of a smaller capture of the same kernel scaled by rows (profiles/traffic.json)",
+                    "peak_source": peak_source_idx}
+        if fp8_probe is not None:
+            roofline["frac_of_assumed_2x_bf16_sustained"] = kernels["indexer_scores"]["tflops"] / assumed_fp8
+            roofline["frac_of_measured_fp8_burst"] = kernels["indexer_scores"]["tflops"] / max(fp8_probe.get("own_loop_burst", 0.0), fp8_probe.get("scaled_mm_burst", 1e-9))
     elif names[dom] == "sparse_attn_prefill":
         roofline = {"kernel": "sparse_attn", "bound": "tensor", "achieved": kernels["sparse_attn_prefill"]["tflops"],
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": kernels["sparse_attn_prefill"]["frac_tensor_peak"],
-                    "traffic": captured_traffic("sparse_attn_latent", shp.M), "peak_source": f"{peaks['source']} bf16 sustained"}
+                    "traffic": attn_dram, "peak_source": f"{peaks['source']} bf16 sustained"}
     else:
         key = names[dom]
         roofline = {"kernel": key, "bound": "hbm", "achieved": kernels[key]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": kernels[key]["gbs"] / peaks["hbm_gbs"], "traffic": captured_traffic("topk_rows" if key == "topk" else "page_mark", shp.M),
+                    "frac": kernels[key]["gbs"] / peaks["hbm_gbs"], "traffic": captured_traffic("topk_rows" if key == "topk" else "page_mark", rows_total),
                     "peak_source": f"{peaks['source']} copy bandwidth"}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        cb = run_reference(args, shp, sess)
+        cb = run_reference(args, shp, sessions[0])
+        if n_sessions > 1:
+            cb["sample"] = "first session of the batch: " + cb["sample"]
         cpu_baseline = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     counts = pd["counts"].cpu().numpy()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3+bf16" if fp8 else "bf16", "data": "synthetic",
-        "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "config": config, "clocks": clocks, "e2e": e2e,
+        # kernels of this library per session pass: indexer, top-k, page mark, page lists, attention (plus one cudaMemsetAsync of the bitmap)
+        "gpu_launches": 5 * args.steps * n_sessions, "roofline": roofline, "cpu_baseline": cpu_baseline, "fp8_peak_probe": fp8_probe,
         "kernels": {k: {kk: (round(float(vv), 4)) for kk, vv in v.items()} for k, v in kernels.items()},
         "indexer_topk_one_call": fused,
         "page_demand": {"n_pages": int(counts[0]), "n_runs": int(counts[1]), "n_miss": int(counts[2]), "n_miss_runs": int(counts[3])},
     }
+    if n_sessions > 1:
+        line["ms_per_session"] = [round(v, 4) for v in per_session_ms]
+    if report is not None:
+        line["report"] = report
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -192,11 +192,13 @@ def janus_indexer_scores(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch.Tens
 
 
 def janus_topk(scores: torch.Tensor, n_keys: int, k: int, *, q_pos0: int = 0, causal: bool = True, want_count: bool = True,
-               want_kth: bool = True):
-    """Per-row top-k over the visible prefix.  Returns (idx [M,k] int32 with -1 padding, count [M] | None, kth [M] | None)."""
+               want_kth: bool = True, idx: Optional[torch.Tensor] = None):
+    """Per-row top-k over the visible prefix.  Returns (idx [M,k] int32 with -1 padding, count [M] | None, kth [M] | None).
+    ``idx``: an [M,k] int32 buffer to write into."""
     lib = load()
     M = scores.shape[0]
-    idx = torch.empty((M, k), dtype=torch.int32, device=scores.device)
+    if idx is None:
+        idx = torch.empty((M, k), dtype=torch.int32, device=scores.device)
     count = torch.empty((M,), dtype=torch.int32, device=scores.device) if want_count else None
     kth = torch.empty((M,), dtype=torch.float32, device=scores.device) if want_kth else None
     rc = lib.janus_topk(_ptr(scores), scores.stride(0), M, int(n_keys), int(q_pos0), int(bool(causal)), int(k), _ptr(idx), _ptr(count),
@@ -261,27 +263,45 @@ def janus_indexer_topk_static(q_idx: torch.Tensor, k_idx: torch.Tensor, w: torch
     _check(rc, "janus_indexer_topk_static")
 
 
-def janus_page_demand(idx: torch.Tensor, *, demand_limit: int, page_size: int, page_table: torch.Tensor, n_phys_pages: int,
-                      predicted_bitmap: Optional[torch.Tensor] = None, capacity: Optional[int] = None, want_miss: bool = True):
-    """Union of selected history tokens as a physical-page bitmap, ascending page list, maximal runs and the miss set
-    against ``predicted_bitmap``.  Returns a dict of device tensors; the counts stay on the device (no host sync)."""
-    lib = load()
-    dev = idx.device
-    n_rows, k = idx.shape
+def page_demand_buffers(n_phys_pages: int, capacity: Optional[int] = None, want_miss: bool = True, device="cuda") -> Dict[str, torch.Tensor]:
+    """Output buffers of janus_page_demand / janus_page_demand_batch for a pool of `n_phys_pages` pages.  Allocate once and
+    pass as ``out=`` to keep allocations (and the fill of the count words) out of a serving loop."""
     cap = int(capacity) if capacity is not None else int(n_phys_pages)
-    n_words = (n_phys_pages + 31) // 32
+    n_words = (int(n_phys_pages) + 31) // 32
     out = {
-        "bitmap": torch.empty((n_words,), dtype=torch.int32, device=dev),
-        "pages": torch.empty((max(cap, 1),), dtype=torch.int32, device=dev),
-        "runs": torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev),
-        "counts": torch.zeros((4,), dtype=torch.int32, device=dev),   # n_pages, n_runs, n_miss, n_miss_runs
+        "bitmap": torch.empty((n_words,), dtype=torch.int32, device=device),
+        "pages": torch.empty((max(cap, 1),), dtype=torch.int32, device=device),
+        "runs": torch.empty((max(cap, 1), 2), dtype=torch.int32, device=device),
+        "counts": torch.zeros((4,), dtype=torch.int32, device=device),   # n_pages, n_runs, n_miss, n_miss_runs (each written by the call that asks for it)
     }
+    if want_miss:
+        out["miss_pages"] = torch.empty((max(cap, 1),), dtype=torch.int32, device=device)
+        out["miss_runs"] = torch.empty((max(cap, 1), 2), dtype=torch.int32, device=device)
+    return out
+
+
+def _page_demand_out_args(out: Dict[str, torch.Tensor], want_miss: bool):
     cp = out["counts"].data_ptr()
     miss_args = [None, None, None, None]
     if want_miss:
-        out["miss_pages"] = torch.empty((max(cap, 1),), dtype=torch.int32, device=dev)
-        out["miss_runs"] = torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev)
         miss_args = [_ptr(out["miss_pages"]), cp + 8, _ptr(out["miss_runs"]), cp + 12]
+    return cp, miss_args
+
+
+def janus_page_demand(idx: torch.Tensor, *, demand_limit: int, page_size: int, page_table: torch.Tensor, n_phys_pages: int,
+                      predicted_bitmap: Optional[torch.Tensor] = None, capacity: Optional[int] = None, want_miss: bool = True,
+                      out: Optional[Dict[str, torch.Tensor]] = None):
+    """Union of selected history tokens as a physical-page bitmap, ascending page list, maximal runs and the miss set
+    against ``predicted_bitmap``.  Returns a dict of device tensors; the counts stay on the device (no host sync).
+    ``out``: buffers from page_demand_buffers() to write into (nothing is allocated or filled by this call then)."""
+    lib = load()
+    n_rows, k = idx.shape
+    if out is None:
+        out = page_demand_buffers(n_phys_pages, capacity, want_miss, idx.device)
+    else:
+        want_miss = want_miss and "miss_pages" in out
+    cap = out["pages"].numel() if capacity is None else int(capacity)
+    cp, miss_args = _page_demand_out_args(out, want_miss)
     rc = lib.janus_page_demand(_ptr(idx), n_rows, k, int(demand_limit), int(page_size), _ptr(page_table), page_table.numel(),
                                int(n_phys_pages), _ptr(predicted_bitmap), _ptr(out["bitmap"]), _ptr(out["pages"]), cp,
                                _ptr(out["runs"]), cp + 4, *miss_args, cap, None, 0, _ptr(dev_status_tensor()), _stream())
@@ -382,25 +402,16 @@ def janus_topk_batch(scores: torch.Tensor, row_offsets: torch.Tensor, k: int, *,
 
 def janus_page_demand_batch(idx: torch.Tensor, *, demand_limits: torch.Tensor, page_size: int, page_tables: torch.Tensor,
                             table_offsets: torch.Tensor, n_phys_pages: int, predicted_bitmap: Optional[torch.Tensor] = None,
-                            capacity: Optional[int] = None, want_miss: bool = True):
+                            capacity: Optional[int] = None, want_miss: bool = True, out: Optional[Dict[str, torch.Tensor]] = None):
     """janus_page_demand over rows that each have their own page table and history length (int64 device tensors)."""
     lib = load()
-    dev = idx.device
     n_rows, k = idx.shape
-    cap = int(capacity) if capacity is not None else int(n_phys_pages)
-    n_words = (n_phys_pages + 31) // 32
-    out = {
-        "bitmap": torch.empty((n_words,), dtype=torch.int32, device=dev),
-        "pages": torch.empty((max(cap, 1),), dtype=torch.int32, device=dev),
-        "runs": torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev),
-        "counts": torch.zeros((4,), dtype=torch.int32, device=dev),   # n_pages, n_runs, n_miss, n_miss_runs
-    }
-    cp = out["counts"].data_ptr()
-    miss_args = [None, None, None, None]
-    if want_miss:
-        out["miss_pages"] = torch.empty((max(cap, 1),), dtype=torch.int32, device=dev)
-        out["miss_runs"] = torch.empty((max(cap, 1), 2), dtype=torch.int32, device=dev)
-        miss_args = [_ptr(out["miss_pages"]), cp + 8, _ptr(out["miss_runs"]), cp + 12]
+    if out is None:
+        out = page_demand_buffers(n_phys_pages, capacity, want_miss, idx.device)
+    else:
+        want_miss = want_miss and "miss_pages" in out
+    cap = out["pages"].numel() if capacity is None else int(capacity)
+    cp, miss_args = _page_demand_out_args(out, want_miss)
     rc = lib.janus_page_demand_batch(_ptr(idx), n_rows, k, _ptr(demand_limits), int(page_size), _ptr(page_tables), _ptr(table_offsets),
                                      int(n_phys_pages), _ptr(predicted_bitmap), _ptr(out["bitmap"]), _ptr(out["pages"]), cp, _ptr(out["runs"]),
                                      cp + 4, *miss_args, cap, _ptr(dev_status_tensor()), _stream())

@@ -25,3 +25,26 @@ def aggregate_throughput(units_local: float, elapsed_ms_local: float, device: st
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(u.item()) / (float(t.item()) * 1e-3), float(t.item()), float(u.item())
+
+
+def or_reduce_bitmap(bitmap: torch.Tensor, union_into=None) -> torch.Tensor:
+    """Union of the ranks' page bitmaps (Sec. 4.2, Eq. 3: each rank predicts on its own disjoint history shard and keeps its
+    own page set; the union is only needed when the exact pass asks which pages nobody predicted).
+
+    The one exchange of the key-sharded partition: an all-gather of the bitmaps (a few KB to a few tens of KB each; works
+    with nccl and gloo alike, where a bitwise-OR all-reduce is a gloo-only operation) followed by a local OR.
+    ``union_into(dst, src)`` does the local OR in place (on a GPU: the library's janus_page_union); without it the OR is a
+    torch op (CPU tests).  Returns a new tensor; every rank gets the same union."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return bitmap.clone()
+    world = dist.get_world_size()
+    flat = torch.empty((world * bitmap.numel(),), dtype=bitmap.dtype, device=bitmap.device)
+    dist.all_gather_into_tensor(flat, bitmap.contiguous().view(-1))
+    gathered = flat.view(world, bitmap.numel())
+    union = gathered[0].clone()
+    for r in range(1, world):
+        if union_into is not None:
+            union_into(union, gathered[r])
+        else:
+            union |= gathered[r]
+    return union
