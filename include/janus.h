@@ -133,6 +133,10 @@ int janus_indexer_topk(const void* q_idx, int64_t q_stride_tok,
                        int64_t q_pos0, int causal, int dtype, int k,
                        int32_t* idx, int32_t* count, float* kth,
                        void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+/* Diagnostic: byte offset inside `ws` of an int32 that holds, after janus_indexer_topk has run, how many rows the sampled
+ * threshold misjudged (they were recomputed exactly, so the result does not depend on it); -1 when this problem takes
+ * the score-matrix route and has no such counter.  Same arguments as janus_indexer_topk_workspace_size. */
+int64_t janus_indexer_topk_fallback_counter_offset(int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal, int dtype, int k);
 
 /*
  * janus_indexer_topk on scratch built into the library - no counterpart in the paper; a convenience of this library.

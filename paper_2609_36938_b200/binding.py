@@ -26,7 +26,7 @@ EXPORTS = [
     "janus_version", "janus_last_cuda_error",
     "janus_indexer_scores_workspace_size", "janus_indexer_scores",
     "janus_topk_workspace_size", "janus_topk",
-    "janus_indexer_topk_workspace_size", "janus_indexer_topk", "janus_indexer_topk_static",
+    "janus_indexer_topk_workspace_size", "janus_indexer_topk", "janus_indexer_topk_static", "janus_indexer_topk_fallback_counter_offset",
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
     "janus_indexer_scores_batch", "janus_topk_batch", "janus_page_demand_batch", "janus_sparse_attn_decode",
@@ -64,6 +64,8 @@ def load() -> ctypes.CDLL:
     lib.janus_topk.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p, c_p]
     lib.janus_indexer_topk_workspace_size.restype = c_sz
     lib.janus_indexer_topk_workspace_size.argtypes = [c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i]
+    lib.janus_indexer_topk_fallback_counter_offset.restype = c_i64
+    lib.janus_indexer_topk_fallback_counter_offset.argtypes = [c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i]
     lib.janus_indexer_topk.restype = c_i
     lib.janus_indexer_topk.argtypes = [c_p, c_i64, c_p, c_i64, c_p, c_p, c_i64, c_p, c_p, c_p, c_i, c_i, c_i, c_i64, c_i64, c_i, c_i, c_i,
                                        c_p, c_p, c_p, c_p, c_sz, c_p, c_p]

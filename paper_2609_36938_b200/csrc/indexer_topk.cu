@@ -262,6 +262,12 @@ extern "C" size_t janus_indexer_topk_workspace_size(int M, int H_I, int D_I, int
     return janus::fused_layout(M, H_I, D_I, n_keys, q_pos0, causal, dtype, k).total;
 }
 
+extern "C" int64_t janus_indexer_topk_fallback_counter_offset(int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal, int dtype, int k) {
+    if (M <= 0 || H_I <= 0 || D_I <= 0 || n_keys <= 0 || k <= 0) return -1;
+    const janus::FusedLayout L = janus::fused_layout(M, H_I, D_I, n_keys, q_pos0, causal, dtype, k);
+    return L.fused ? static_cast<int64_t>(L.fb_count) : -1;
+}
+
 extern "C" int janus_indexer_topk(const void* q_idx, int64_t q_stride_tok, const void* k_idx, int64_t k_stride_tok, const float* w,
                                   const float* q_scale, int64_t q_scale_stride_tok, const float* k_scale, const float* row_bias,
                                   const float* col_bias, int M, int H_I, int D_I, int64_t n_keys, int64_t q_pos0, int causal, int dtype,

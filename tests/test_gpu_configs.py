@@ -42,6 +42,18 @@ def oracle_row_scores(sess, t, *, predicted=False):
                             recency=sess["recency"], q_pos0=shp.L + t, causal=True)[0]
 
 
+def boundary_rows(shp):
+    """Query rows whose causal diagonal (their own key, position L + t) is the last key of a 128-key tile and the first key
+    of the next one, the same for the 64-tile key chunk one CTA of the indexer walks (8192 keys), and the last and first
+    row of a CTA's 16-token query group: the places where a tile-edge or mask-edge mistake would show."""
+    rows = set()
+    for period in (128, 64 * 128):
+        t_last = (period - 1 - shp.L) % period           # L + t = period - 1 (mod period)
+        rows |= {t_last, t_last + 1}
+    rows |= {15, 16}
+    return np.array(sorted(t for t in rows if 0 <= t < shp.M), dtype=np.int64)
+
+
 def run_and_check(sess, n_rows=N_SAMPLE_ROWS):
     shp = sess["shape"]
     d = Hp.upload_session(sess)
@@ -65,7 +77,7 @@ def run_and_check(sess, n_rows=N_SAMPLE_ROWS):
                                            softmax_scale=shp.softmax_scale, d_v=shp.d_v)
     B.check_dev_status()
 
-    rows = W.sample_rows(shp.M, n_rows)
+    rows = np.unique(np.concatenate([W.sample_rows(shp.M, n_rows), boundary_rows(shp)]))
     idx_np = idx.cpu().numpy()
     # ---- properties on every row
     cnt = count.cpu().numpy()

@@ -2,6 +2,8 @@
 Checked against janus_indexer_topk (caller's workspace) on the same inputs, twice in a row (the second call runs on
 whatever the first left in the array), on a shape that takes the candidate-list route and one that takes the two-call
 route; the device's free memory must not move across the calls; a problem beyond the array is refused.
+The comparator is the library's own workspace call, not the oracle: that call's oracle check lives in
+tests/test_gpu_fused.py and tests/test_gpu_fullsize.py, so agreement with it carries the oracle check over to this entry.
 The file name sorts last on purpose: the array has then been used by nothing, or by anything, before."""
 import numpy as np
 import pytest
