@@ -147,9 +147,8 @@ def captured_traffic(kernel_key: str, rows: int):
     p = os.path.join(ROOT, "profiles", "traffic.json")
     if not os.path.exists(p):
         return None
-    d = json.load(open(p))
-    b = d.get("dram_bytes_per_launch", {}).get(kernel_key)
-    return None if b is None else b * rows / d["rows_in_capture"]
+    e = json.load(open(p)).get("dram_bytes_per_launch", {}).get(kernel_key)
+    return None if e is None else e["bytes"] * rows / e["rows"]
 
 
 def workload_numbers(shp):
