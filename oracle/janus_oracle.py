@@ -178,6 +178,24 @@ def entry_visible_prefix(t: int, n_entries: int, q_pos0: int, entry_size: int) -
     return max(0, min(n_entries, (q_pos0 + t) // entry_size + 1))
 
 
+def entry_pool_scores(scores, *, entry_size: int, q_pos0: int = 0, causal: bool = True) -> np.ndarray:
+    """Second reading of the entry-granularity footnote of Sec. 2.2 (the paper defines neither): the indexer scores tokens as
+    usual and an entry's score is the maximum over the tokens of the entry that the row may see,
+        entry_score[t, e] = max { score[t, s] : e*E <= s < (e+1)*E, s <= q_pos0 + t },
+    -inf for an entry without a visible token.  scores [n_rows, n_keys]; returns float64 [n_rows, ceil(n_keys / E)]."""
+    scores = np.asarray(scores, dtype=np.float64)
+    n_rows, n_keys = scores.shape
+    n_entries = (n_keys + entry_size - 1) // entry_size
+    out = np.full((n_rows, n_entries), NEG_INF, dtype=np.float64)
+    for t in range(n_rows):
+        prefix = visible_prefix(t, n_keys, q_pos0, causal)
+        for e in range(n_entries):
+            a, b = e * entry_size, min((e + 1) * entry_size, prefix)
+            if b > a:
+                out[t, e] = scores[t, a:b].max()
+    return out
+
+
 def entry_topk(entry_scores, k_e: int, *, q_pos0: int, entry_size: int) -> np.ndarray:
     """Row-wise top-k_e over entries.  Returns int64 [n_rows, k_e] padded with -1."""
     entry_scores = np.asarray(entry_scores)

@@ -500,3 +500,32 @@ def test_e2m1_decode_table_and_packing_order():
     a = O.indexer_scores(q, packed, w, dtype="fp8+fp4k", q_scale=qs, k_scale=ks, causal=False)
     b = O.indexer_scores(q, k8, w, dtype="fp8", q_scale=qs, k_scale=ks, causal=False)
     assert np.array_equal(a, b)
+
+
+def test_entry_pooled_scores_hand_case_and_invariants():
+    # pooled reading of the entry footnote (Sec. 2.2): an entry scores as its best visible token
+    sc = np.array([[1.0, 5.0, -2.0, 0.5, 9.0, 3.0, 7.0],
+                   [4.0, -1.0, 6.0, 2.0, 8.0, 0.0, -3.0]])
+    # E = 3, q_pos0 = 3: row 0 sees tokens 0..3, row 1 sees 0..4
+    got = O.entry_pool_scores(sc, entry_size=3, q_pos0=3, causal=True)
+    assert np.array_equal(got, np.array([[5.0, 0.5, -np.inf], [6.0, 8.0, -np.inf]]))
+    # not causal: every token counts, the last entry is partial
+    assert np.array_equal(O.entry_pool_scores(sc, entry_size=3, causal=False), np.array([[5.0, 9.0, 7.0], [6.0, 8.0, -3.0]]))
+    # E = 1 is the token score itself on the visible prefix
+    rng = np.random.default_rng(31)
+    r = rng.standard_normal((5, 23))
+    one = O.entry_pool_scores(r, entry_size=1, q_pos0=10, causal=True)
+    for t in range(5):
+        assert np.array_equal(one[t, :11 + t], r[t, :11 + t]) and np.all(np.isneginf(one[t, 11 + t:]))
+    # the best entry holds the best visible token; the number of finite entries is the number of entries with a visible token
+    E = 4
+    pooled = O.entry_pool_scores(r, entry_size=E, q_pos0=10, causal=True)
+    for t in range(5):
+        prefix = 11 + t
+        assert int(np.argmax(pooled[t])) == int(np.argmax(r[t, :prefix])) // E
+        assert np.isfinite(pooled[t]).sum() == O.entry_visible_prefix(t, pooled.shape[1], 10, E)
+    # brute force: a sorted copy of each entry's visible tokens ends with the pooled value
+    for t in range(5):
+        for e in range(pooled.shape[1]):
+            vis = [r[t, s] for s in range(e * E, min((e + 1) * E, 23)) if s <= 10 + t]
+            assert pooled[t, e] == (sorted(vis)[-1] if vis else -np.inf)
