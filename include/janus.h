@@ -259,12 +259,21 @@ int janus_sparse_attn_prefill(const void* q, int M, int H_q, int d_qk,
  *                        before position q_pos0 + t, else -1 ([M, k_e * entry_size] int32).  The result feeds
  *                        janus_page_demand and janus_sparse_attn_prefill like any token selection.
  *
+ *   janus_entry_pool_scores   the other reading of the same footnote: the indexer scores tokens as usual and an entry's
+ *                        score is the maximum over its tokens that the row may see,
+ *                            entry_scores[t, e] = max { scores[t, s] : e*E <= s < (e+1)*E, s <= q_pos0 + t }   (causal;
+ *                            every token of the entry otherwise), -inf for an entry without a visible token.
+ *                        scores [M, scores_ld] fp32 from janus_indexer_scores; entry_scores [M, entry_ld] fp32 out,
+ *                        entry_ld >= ceil(n_keys / entry_size) (a multiple of 4 if janus_topk_entries follows).
+ *
  * A selection shared by a group of layers (index reuse) needs no call of its own: pass the same idx to the attention of
  * every layer of the group.
  */
 int janus_topk_entries(const float* scores, int64_t scores_ld, int M, int64_t n_entries,
                        int64_t q_pos0, int entry_size, int k,
                        int32_t* idx, int32_t* count, float* kth, int32_t* dev_status, void* stream);
+int janus_entry_pool_scores(const float* scores, int64_t scores_ld, int M, int64_t n_keys, int64_t q_pos0, int causal,
+                            int entry_size, float* entry_scores, int64_t entry_ld, void* stream);
 int janus_entry_expand(const int32_t* idx_entries, int M, int k_e, int entry_size, int64_t q_pos0,
                        int32_t* idx_tokens, void* stream);
 

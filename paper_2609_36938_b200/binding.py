@@ -30,7 +30,7 @@ EXPORTS = [
     "janus_page_demand_workspace_size", "janus_page_demand", "janus_page_union",
     "janus_sparse_attn_prefill_workspace_size", "janus_sparse_attn_prefill",
     "janus_indexer_scores_batch", "janus_topk_batch", "janus_page_demand_batch", "janus_sparse_attn_decode",
-    "janus_topk_entries", "janus_entry_expand",
+    "janus_topk_entries", "janus_entry_expand", "janus_entry_pool_scores",
     "janus_selftest_bounded_wait", "janus_fp8_mma_probe",
 ]
 
@@ -96,6 +96,8 @@ def load() -> ctypes.CDLL:
                                              c_p, c_p]
     lib.janus_topk_entries.restype = c_i
     lib.janus_topk_entries.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_p, c_p, c_p, c_p]
+    lib.janus_entry_pool_scores.restype = c_i
+    lib.janus_entry_pool_scores.argtypes = [c_p, c_i64, c_i, c_i64, c_i64, c_i, c_i, c_p, c_i64, c_p]
     lib.janus_entry_expand.restype = c_i
     lib.janus_entry_expand.argtypes = [c_p, c_i, c_i, c_i, c_i64, c_p, c_p]
     lib.janus_selftest_bounded_wait.restype = c_i
@@ -352,6 +354,17 @@ def janus_topk_entries(scores: torch.Tensor, n_entries: int, k: int, *, q_pos0: 
                                 _ptr(count), _ptr(kth), _ptr(dev_status_tensor()), _stream())
     _check(rc, "janus_topk_entries")
     return idx, count, kth
+
+
+def janus_entry_pool_scores(scores: torch.Tensor, n_keys: int, *, entry_size: int, q_pos0: int = 0, causal: bool = True) -> torch.Tensor:
+    """Entry scores as the maximum over each entry's visible token scores.  Returns [M, ld] fp32, ld = n_entries rounded up to 4."""
+    M = scores.shape[0]
+    n_entries = (int(n_keys) + entry_size - 1) // entry_size
+    ld = max(4, (n_entries + 3) // 4 * 4)
+    out = torch.empty((M, ld), dtype=torch.float32, device=scores.device)
+    _check(load().janus_entry_pool_scores(_ptr(scores), scores.stride(0), M, int(n_keys), int(q_pos0), int(bool(causal)), int(entry_size),
+                                          _ptr(out), ld, _stream()), "janus_entry_pool_scores")
+    return out
 
 
 def janus_entry_expand(idx_entries: torch.Tensor, *, q_pos0: int, entry_size: int) -> torch.Tensor:

@@ -69,6 +69,29 @@ __global__ void entry_expand_kernel(const int32_t* __restrict__ idx_e, int M, in
     }
 }
 
+// Pooled entry scores (the second reading of the entry footnote of Sec. 2.2): an entry scores as the best of its tokens the
+// row may see.  One warp per (row, entry) strip: lanes read consecutive floats (coalesced), a warp shuffle takes the maximum.
+__global__ void __launch_bounds__(256)
+entry_pool_kernel(const float* __restrict__ scores, int64_t ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int entry_size,
+                  int64_t n_entries, float* __restrict__ out, int64_t out_ld) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_id = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    const float neg_inf = __int_as_float(0xff800000);
+    for (int64_t item = warp_id; item < static_cast<int64_t>(M) * n_entries; item += n_warps) {
+        const int64_t t = item / n_entries, e = item - t * n_entries;
+        const int64_t prefix = causal ? (n_keys < q_pos0 + t + 1 ? n_keys : q_pos0 + t + 1) : n_keys;
+        const int64_t a = e * entry_size;
+        const int64_t b = a + entry_size < prefix ? a + entry_size : prefix;
+        const float* row = scores + t * ld;
+        float m = neg_inf;
+        for (int64_t s = a + lane; s < b; s += 32) m = fmaxf(m, __ldg(row + s));
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        if (lane == 0) out[t * out_ld + e] = m;
+    }
+}
+
 // Batch form (decode over many sessions): row b starts at scores[row_offsets[b]] and has row_lengths[b] elements (or runs
 // up to the next row's start when row_lengths is NULL), every element visible.
 template <int CAP>
@@ -109,6 +132,23 @@ extern "C" int janus_topk_entries(const float* scores, int64_t scores_ld, int M,
     const size_t smem = sizeof(TopkSharedT<TK_CAP>);
     JANUS_CUDA_CHECK(cudaFuncSetAttribute(topk_entries_kernel<TK_CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     topk_entries_kernel<TK_CAP><<<M, TK_THREADS, smem, stream>>>(scores, scores_ld, M, n_entries, q_pos0, entry_size, k, idx, count, kth);
+    JANUS_CUDA_CHECK(cudaGetLastError());
+    return JANUS_OK;
+}
+
+extern "C" int janus_entry_pool_scores(const float* scores, int64_t scores_ld, int M, int64_t n_keys, int64_t q_pos0, int causal, int entry_size,
+                                       float* entry_scores, int64_t entry_ld, void* stream_) {
+    using namespace janus;
+    if (M < 0 || n_keys < 0 || q_pos0 < 0 || entry_size <= 0 || scores_ld < n_keys) return JANUS_ERR_INVALID_ARG;
+    const int64_t n_entries = (n_keys + entry_size - 1) / entry_size;
+    if (entry_ld < n_entries) return JANUS_ERR_INVALID_ARG;
+    if (M == 0 || n_entries == 0) return JANUS_OK;
+    if (!scores || !entry_scores) return JANUS_ERR_INVALID_ARG;
+    const int64_t items = static_cast<int64_t>(M) * n_entries;
+    int64_t blocks = (items + 7) / 8;                        // eight warps per block, one strip each
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    entry_pool_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream_)>>>(scores, scores_ld, M, n_keys, q_pos0, causal,
+                                                                                                    entry_size, n_entries, entry_scores, entry_ld);
     JANUS_CUDA_CHECK(cudaGetLastError());
     return JANUS_OK;
 }

@@ -126,6 +126,10 @@ def test_batch_entry_and_static_entry_validation(lib):
     assert lib.janus_topk_entries(fake, 64, 4, 64, 0, 0, 8, fake, None, None, None, None) == INVALID       # entry_size = 0
     assert lib.janus_topk_entries(fake, 32, 4, 64, 0, 16, 8, fake, None, None, None, None) == INVALID      # ld < n_entries
     assert lib.janus_entry_expand(None, 4, 8, 16, 0, fake, None) == INVALID
+    assert lib.janus_entry_pool_scores(fake, 256, 4, 256, 0, 1, 0, fake, 16, None) == INVALID               # entry_size = 0
+    assert lib.janus_entry_pool_scores(fake, 256, 4, 256, 0, 1, 64, fake, 3, None) == INVALID               # entry_ld < n_entries
+    assert lib.janus_entry_pool_scores(fake, 256, 4, 256, 0, 1, 64, None, 4, None) == INVALID               # no output
+    assert lib.janus_entry_pool_scores(fake, 256, 0, 256, 0, 1, 64, fake, 4, None) == 0                     # M = 0
     assert lib.janus_entry_expand(fake, 0, 8, 16, 0, fake, None) == 0
     # built-in scratch: the size check comes before the device is touched
     assert lib.janus_indexer_topk_static(fake, 64 * 128, fake, 128, fake, fake, 0, fake, None, None, 4096, 64, 128, 135168, 131072, 1, 1, 2048,

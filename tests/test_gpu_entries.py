@@ -80,3 +80,43 @@ def test_selecting_every_entry_is_dense_causal_attention():
     for t in range(M):
         assert sorted(x for x in idx_t[t] if x >= 0) == list(range(L + t + 1))
     B.check_dev_status()
+
+
+@pytest.mark.parametrize("E,L,M,k_e,dtype", [(128, 30000, 20, 12, "bf16"), (16, 2011, 33, 25, "fp8"), (64, 50, 70, 4, "bf16")])
+def test_pooled_entry_scores_pipeline_matches_oracle(E, L, M, k_e, dtype):
+    """The other reading of the entry footnote (Sec. 2.2): token scores from the ordinary indexer, an entry scores as the
+    maximum over its visible tokens (janus_entry_pool_scores), then the same entry top-k and expansion."""
+    rng = np.random.default_rng(7 * E + L)
+    S = L + M
+    n_entries = (S + E - 1) // E
+    H, D = 64, 128
+    qf, kf = rng.standard_normal((M, H, D)).astype(np.float32), rng.standard_normal((S, D)).astype(np.float32)
+    w = (rng.uniform(0, 1, (M, H)) / 8).astype(np.float32)
+    if dtype == "bf16":
+        q, kk, qs, ks = W.to_bf16_bits(qf), W.to_bf16_bits(kf), None, None
+    else:
+        q, kk = W.to_e4m3_bits(2 * qf), W.to_e4m3_bits(2 * kf)
+        qs, ks = np.exp2(rng.uniform(-2, 2, H)).astype(np.float32), np.exp2(rng.uniform(-1, 1, S)).astype(np.float32)
+    sc = B.janus_indexer_scores(dev(q, dtype), dev(kk, dtype), dev(w, "f32"), q_scale=dev(qs, "f32"), k_scale=dev(ks, "f32"), q_pos0=L, causal=True)
+    pooled = B.janus_entry_pool_scores(sc, S, entry_size=E, q_pos0=L, causal=True)
+    idx_e, cnt, _ = B.janus_topk_entries(pooled, n_entries, k_e, q_pos0=L, entry_size=E)
+    idx_t = B.janus_entry_expand(idx_e, q_pos0=L, entry_size=E)
+    B.check_dev_status()
+    # pooling is a maximum of fp32 values: exact on the library's own scores
+    sc_h = sc[:, :S].cpu().numpy()
+    want_pooled = O.entry_pool_scores(sc_h, entry_size=E, q_pos0=L, causal=True)
+    assert np.array_equal(pooled[:, :n_entries].cpu().numpy().astype(np.float64), want_pooled)
+    # against the oracle's own scores: entry selection within the 1e-3 band, expansion exact
+    ref_sc = O.indexer_scores(q, kk, w, dtype=dtype, q_scale=qs, k_scale=ks, q_pos0=L, causal=True)
+    ref_pooled = O.entry_pool_scores(ref_sc, entry_size=E, q_pos0=L, causal=True)
+    idx_e_h = idx_e.cpu().numpy()
+    for t in range(M):
+        prefix = O.entry_visible_prefix(t, n_entries, L, E)
+        assert cnt.cpu().numpy()[t] == min(k_e, prefix)
+        ok, msg = O.topk_row_agrees(idx_e_h[t], ref_pooled[t], prefix, k_e)
+        assert ok, f"row {t}: {msg}"
+    assert np.array_equal(idx_t.cpu().numpy(), O.entry_expand(idx_e_h, q_pos0=L, entry_size=E))
+    # non-causal pooling (the prediction pass over history keys only)
+    nc = B.janus_entry_pool_scores(sc, L, entry_size=E, causal=False)
+    assert np.array_equal(nc[:, :(L + E - 1) // E].cpu().numpy().astype(np.float64), O.entry_pool_scores(sc_h[:, :L], entry_size=E, causal=False))
+    B.check_dev_status()
