@@ -370,6 +370,92 @@ def run_sharded_prediction(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_query_sharded(args, rank, world, local_rank):
+    """--shard queries: the query-parallel partition (Sec. 4.2): query rows are independent, so rank n runs the whole exact
+    pass (indexer -> top-k -> page demand -> attention) on its contiguous slice of the M new tokens against replicated keys and
+    KV pool; the only exchange is the union of the ranks' page bitmaps (one all-gather + janus_page_union), from which every
+    rank has the session's page demand.  Total work is fixed: strong scaling."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_36938_b200 import binding as B, build as _build, dist_utils as D, workloads as W
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    B.load()
+    shp = W.config_shape(args.workload if args.workload != 4 else 3, L=args.L, M=args.M)
+    sess = W.make_session(shp, args.seed)                      # the same session on every rank
+    kind = shp.idx_dtype
+    r0, r1 = rank * shp.M // world, (rank + 1) * shp.M // world
+    m = r1 - r0
+    n_keys = shp.L + r1                                        # keys the last row of the slice may see
+    dev = lambda name, kd, sl=slice(None): None if sess[name] is None else B.to_device(sess[name][sl], kd)
+    q_idx, w, Q = dev("q_idx", kind, slice(r0, r1)), dev("w", "f32", slice(r0, r1)), dev("Q", "bf16", slice(r0, r1))
+    k_idx, k_scale, col_bias = dev("k_idx", kind, slice(0, n_keys)), dev("k_scale", "f32", slice(0, n_keys)), dev("col_bias", "f32", slice(0, n_keys))
+    q_scale, row_bias = dev("q_scale", "f32"), dev("row_bias", "f32", slice(r0, r1))
+    table, pool = dev("page_table", "i32"), dev("k_pool", "bf16")
+    n_phys = sess["n_phys_pages"]
+    ld = (n_keys + 31) // 32 * 32
+    scores = torch.empty((max(m, 1), ld), dtype=torch.float32, device="cuda")
+    idx = torch.empty((max(m, 1), shp.k), dtype=torch.int32, device="cuda")
+    out = torch.empty((max(m, 1), shp.H_q, shp.d_v), dtype=torch.bfloat16, device="cuda")
+    bufs = B.page_demand_buffers(n_phys, want_miss=False)
+    union_fn = lambda dst, src: B.janus_page_union(dst, src, n_phys)
+
+    def step():
+        if m > 0:
+            sc = B.janus_indexer_scores(q_idx, k_idx, w, q_scale=q_scale, k_scale=k_scale, row_bias=row_bias, col_bias=col_bias, q_pos0=shp.L + r0,
+                                        causal=True, scores=scores)
+            B.janus_topk(sc, n_keys, shp.k, q_pos0=shp.L + r0, causal=True, want_count=False, want_kth=False, idx=idx)
+            pd = B.janus_page_demand(idx, demand_limit=shp.L, page_size=shp.page_size, page_table=table, n_phys_pages=n_phys, want_miss=False, out=bufs)
+            B.janus_sparse_attn_prefill(Q, pool, pool, idx, page_table=table, page_size=shp.page_size, softmax_scale=shp.softmax_scale, d_v=shp.d_v,
+                                        want_lse=False, out=out)
+            bm = pd["bitmap"]
+        else:
+            bm = torch.zeros_like(bufs["bitmap"])
+        return D.or_reduce_bitmap(bm, union_fn)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        sampler.wait_until_running()
+    for _ in range(max(args.warmup, 3)):
+        union = step()
+    B.check_dev_status()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        union = step()
+    e1.record()
+    barrier()
+    B.check_dev_status()
+    value, elapsed_ms, _ = D.aggregate_throughput(float(shp.M * args.steps) if rank == 0 else 0.0, e0.elapsed_time(e1), device="cuda")
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        from paper_2609_36938_b200 import report as R
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                "dtype": "fp8_e4m3+bf16" if kind == "fp8" else "bf16", "data": "synthetic", "clocks": clocks,
+                "config": {"workload": f"query-sharded exact pass: L={shp.L} M={shp.M} k={shp.k} split into {world} contiguous row slices, keys and KV pool "
+                                       f"replicated, indexer {shp.H_I}x{shp.D_I} {kind}, latent attention, page {shp.page_size}",
+                           "exchange": "one all-gather of the page bitmaps + local union (janus_page_union) per step"},
+                "gpu_launches": 5 * args.steps, "union_pages": R.popcount(union)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -387,8 +473,9 @@ def main():
     ap.add_argument("--no-fused", action="store_true", help="skip the side measurement of janus_indexer_topk")
     ap.add_argument("--no-peak-probe", action="store_true", help="skip the FP8 tensor-rate probe (the roofline then divides by an assumed peak)")
     ap.add_argument("--no-report", action="store_true", help="skip the recall / precision / run-length report of configs 1, 4, 5")
-    ap.add_argument("--shard", default="none", choices=["none", "keys"],
-                    help="keys: with --gpus N, time the key-sharded prediction pass (Eq. 3): rank n scores its own history shard")
+    ap.add_argument("--shard", default="none", choices=["none", "keys", "queries"],
+                    help="with --gpus N: keys = time the key-sharded prediction pass (Eq. 3): rank n scores its own history shard; "
+                         "queries = rank n runs the exact pass on its slice of the new tokens; either way one union of page bitmaps")
     ap.add_argument("--decode-batch", type=int, default=0, help="side workload: time one decode step over this many sessions instead")
     ap.add_argument("--decode-fp4-keys", action="store_true", help="with --decode-batch: indexer keys stored as FP4 E2M1")
     args = ap.parse_args()
@@ -404,6 +491,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.shard == "keys" and args.impl == "ours":
         run_sharded_prediction(args, rank, world, local_rank)
+        return
+    if args.shard == "queries" and args.impl == "ours":
+        run_query_sharded(args, rank, world, local_rank)
         return
 
     from paper_2609_36938_b200 import workloads as W

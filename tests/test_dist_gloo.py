@@ -130,3 +130,36 @@ def test_or_reduce_bitmap_single_process_passthrough():
     b = torch.tensor([5, 0, -1], dtype=torch.int32)
     u = D.or_reduce_bitmap(b)
     assert torch.equal(u, b) and u.data_ptr() != b.data_ptr()
+
+
+# ---- query-parallel partition (Sec. 4.2): each rank selects for its slice of the new tokens, the page sets are united -----------
+def _query_worker(rank, world, port, out):
+    from oracle import janus_oracle as O
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        shp, sess = _shard_session()
+        r0, r1 = rank * shp.M // world, (rank + 1) * shp.M // world
+        sc = O.indexer_scores(sess["q_idx"], sess["k_idx"], sess["w"], dtype=shp.idx_dtype, q_pos0=shp.L, causal=True, rows=range(r0, r1))
+        idx = O.topk(sc, shp.k, q_pos0=shp.L, causal=True, rows=range(r0, r1))
+        mine = O.page_demand(idx, shp.L, shp.page_size, sess["page_table"])["pages"]
+        union = D.or_reduce_bitmap(_pages_to_bitmap(mine, sess["n_phys_pages"]))
+        out[rank] = (mine, _bitmap_to_pages(union, sess["n_phys_pages"]))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_split_the_query_rows_and_unite_their_page_sets():
+    from oracle import janus_oracle as O
+
+    world = 2
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_query_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+    shp, sess = _shard_session()
+    sc = O.indexer_scores(sess["q_idx"], sess["k_idx"], sess["w"], dtype=shp.idx_dtype, q_pos0=shp.L, causal=True)
+    full = O.page_demand(O.topk(sc, shp.k, q_pos0=shp.L, causal=True), shp.L, shp.page_size, sess["page_table"])["pages"]
+    (mine0, union0), (mine1, union1) = out[0], out[1]
+    assert union0 == union1 == full == sorted(set(mine0) | set(mine1))      # rows are independent: the union is the session's demand
