@@ -507,7 +507,8 @@ int launch_indexer_tc(const void* q_idx, const void* k_idx, int64_t k_stride_tok
     const int n_groups = (M + tpc - 1) / tpc;
     int64_t per = (static_cast<int64_t>(p.n_tiles) * n_groups + 148 * 4 - 1) / (148 * 4);
     if (per < 2) per = 2;
-    if (per > 64) per = 64;
+    if (per > (cand_mode ? 64 : 256)) per = cand_mode ? 64 : 256;     // a CTA's start-up (query tile load, tensor-memory allocation) is paid once per `per` key tiles:
+                                  // 256 against 64 was 1-2 % at 131072 keys x 4096 rows, with still about seven waves of CTAs
     p.tiles_per_cta = static_cast<int>(per);
     dim3 grid((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, n_groups);
     if (grid.y > 65535) return JANUS_ERR_UNSUPPORTED;

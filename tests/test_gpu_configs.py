@@ -44,10 +44,10 @@ def oracle_row_scores(sess, t, *, predicted=False):
 
 def boundary_rows(shp):
     """Query rows whose causal diagonal (their own key, position L + t) is the last key of a 128-key tile and the first key
-    of the next one, the same for the 64-tile key chunk one CTA of the indexer walks (8192 keys), and the last and first
+    of the next one, the same for the key chunk one CTA of the indexer walks (up to 256 tiles; 64 tiles checked too), and the last and first
     row of a CTA's 16-token query group: the places where a tile-edge or mask-edge mistake would show."""
     rows = set()
-    for period in (128, 64 * 128):
+    for period in (128, 64 * 128, 256 * 128):
         t_last = (period - 1 - shp.L) % period           # L + t = period - 1 (mod period)
         rows |= {t_last, t_last + 1}
     rows |= {15, 16}
